@@ -1,0 +1,317 @@
+"""Pins for the fp64 oracle: each test ties it to something fixed outside the oracle itself -
+library attention and autograd (torch CPU, fp64), closed forms, finite differences, the
+paper's cost model and its gradient-reach statements.  No GPU is used here."""
+import os
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+import oracle
+from oracle import dense
+
+RNG = np.random.default_rng(7)
+TOL = 1e-10
+
+
+def rand(B, L, Hq, Hkv, d, rng=RNG):
+    return (rng.standard_normal((B, L, Hq, d)), rng.standard_normal((B, L, Hkv, d)),
+            rng.standard_normal((B, L, Hkv, d)), rng.standard_normal((B, L, Hq, d)))
+
+
+def t64(a, grad=False):
+    return torch.tensor(a, dtype=torch.float64, requires_grad=grad)
+
+
+def sdpa_causal(Q, K, V, dO):
+    """Textbook full causal attention and its gradients from the library (fp64), with GQA expansion."""
+    q, k, v = t64(Q, True), t64(K, True), t64(V, True)
+    g = Q.shape[2] // K.shape[2]
+    kk = k.repeat_interleave(g, dim=2)
+    vv = v.repeat_interleave(g, dim=2)
+    o = F.scaled_dot_product_attention(q.transpose(1, 2), kk.transpose(1, 2), vv.transpose(1, 2), is_causal=True)
+    o = o.transpose(1, 2)
+    (o * t64(dO)).sum().backward()
+    s = torch.einsum("blhd,bmhd->bhlm", q, kk) / np.sqrt(Q.shape[3])
+    L = Q.shape[1]
+    s = s.masked_fill(~torch.ones(L, L, dtype=torch.bool).tril(), float("-inf"))
+    lse = torch.logsumexp(s, dim=-1)
+    return o.detach().numpy(), lse.detach().numpy(), q.grad.numpy(), k.grad.numpy(), v.grad.numpy()
+
+
+# ---- forward / backward: S >= L is textbook causal attention --------------------------------
+@pytest.mark.parametrize("S,T", [(64, 0), (64, 64), (200, 17)])
+def test_single_segment_equals_library_causal_attention(S, T):
+    Q, K, V, dO = rand(2, 64, 4, 2, 16)
+    o, lse, gq, gk, gv = sdpa_causal(Q, K, V, dO)
+    O, LSE = oracle.fwd(Q, K, V, S, T)
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, T)
+    for a, b in ((O, o), (LSE, lse), (dQ, gq), (dK, gk), (dV, gv)):
+        np.testing.assert_allclose(a, b, rtol=0, atol=TOL)
+
+
+def test_no_tail_no_flags_is_block_diagonal():
+    S, L = 24, 96
+    Q, K, V, dO = rand(1, L, 2, 2, 8)
+    O, LSE = oracle.fwd(Q, K, V, S, 0)
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, 0)
+    for i in range(L // S):
+        sl = slice(i * S, (i + 1) * S)
+        o, lse, gq, gk, gv = sdpa_causal(Q[:, sl], K[:, sl], V[:, sl], dO[:, sl])
+        np.testing.assert_allclose(O[:, sl], o, atol=TOL)
+        np.testing.assert_allclose(LSE[:, :, sl], lse, atol=TOL)
+        np.testing.assert_allclose(dQ[:, sl], gq, atol=TOL)
+        np.testing.assert_allclose(dK[:, sl], gk, atol=TOL)
+        np.testing.assert_allclose(dV[:, sl], gv, atol=TOL)
+
+
+@pytest.mark.parametrize("S,T", [(16, 0), (16, 5), (32, 32), (7, 3)])
+def test_all_heads_flagged_forward_is_full_causal(S, T):
+    Q, K, V, dO = rand(1, 80, 4, 2, 8)
+    o, lse, gq, _, _ = sdpa_causal(Q, K, V, dO)
+    O, LSE = oracle.fwd(Q, K, V, S, T, head_past_mask=[1, 1])
+    np.testing.assert_allclose(O, o, atol=TOL)
+    np.testing.assert_allclose(LSE, lse, atol=TOL)
+    # stop-gradient cuts K/V only: dQ is the full-causal dQ
+    dQ, _, _ = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=[1, 1])
+    np.testing.assert_allclose(dQ, gq, atol=TOL)
+
+
+# ---- the paper's segment recurrence, built with library ops and autograd -----------------------
+def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False):
+    """For every segment i and head: context = [sg(older past) if flagged ; tail of segment i-1 ;
+    own segment], every prefix position visible and the own segment causal (Appendix C), run
+    through library attention; stop-gradient realised with .detach() (Definition 3.2)."""
+    q, k, v = t64(Q, True), t64(K, True), t64(V, True)
+    B, L, Hq, d = Q.shape
+    Hkv = K.shape[2]
+    g = Hq // Hkv
+    outs = torch.zeros(B, L, Hq, d, dtype=torch.float64)
+    lses = torch.zeros(B, Hq, L, dtype=torch.float64)
+    pieces = []
+    for i in range((L + S - 1) // S):
+        s0, s1 = i * S, min(L, (i + 1) * S)
+        a = max(0, s0 - T)
+        for h in range(Hq):
+            c = h // g
+            ks, vs = [], []
+            if flags[c] and a > 0:
+                ks.append(k[:, :a, c].detach())
+                vs.append(v[:, :a, c].detach())
+            if s0 > a:
+                kt, vt = k[:, a:s0, c], v[:, a:s0, c]
+                if flags[c] and flagged_tail_is_sg:
+                    kt, vt = kt.detach(), vt.detach()
+                ks.append(kt)
+                vs.append(vt)
+            ks.append(k[:, s0:s1, c])
+            vs.append(v[:, s0:s1, c])
+            kc, vc = torch.cat(ks, dim=1), torch.cat(vs, dim=1)
+            P = kc.shape[1] - (s1 - s0)
+            m = torch.ones(s1 - s0, kc.shape[1], dtype=torch.bool)
+            m[:, P:] = torch.ones(s1 - s0, s1 - s0, dtype=torch.bool).tril()
+            o = F.scaled_dot_product_attention(q[:, s0:s1, h].unsqueeze(1), kc.unsqueeze(1), vc.unsqueeze(1),
+                                               attn_mask=m).squeeze(1)
+            pieces.append((o * t64(dO[:, s0:s1, h])).sum())
+            outs[:, s0:s1, h] = o.detach()
+            sc = torch.einsum("bld,bmd->blm", q[:, s0:s1, h], kc) / np.sqrt(d)
+            lses[:, h, s0:s1] = torch.logsumexp(sc.masked_fill(~m, float("-inf")), dim=-1).detach()
+    torch.stack(pieces).sum().backward()
+    return outs.numpy(), lses.numpy(), q.grad.numpy(), k.grad.numpy(), v.grad.numpy()
+
+
+@pytest.mark.parametrize("L,S,T,flags,variant", [
+    (96, 32, 8, [0, 1], False),
+    (96, 32, 32, [1, 0], False),
+    (100, 32, 8, [0, 1], False),      # ragged last segment
+    (90, 30, 7, [1, 1], False),
+    (96, 32, 8, [0, 1], True),        # flagged heads' tail reads stop-gradient too
+    (64, 16, 0, [0, 0], False),
+])
+def test_segment_recurrence_with_autograd(L, S, T, flags, variant):
+    Q, K, V, dO = rand(2, L, 4, 2, 8)
+    o, lse, gq, gk, gv = recurrence_autograd(Q, K, V, dO, S, T, flags, variant)
+    O, LSE = oracle.fwd(Q, K, V, S, T, head_past_mask=flags)
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=flags, flagged_tail_is_sg=variant)
+    np.testing.assert_allclose(O, o, atol=TOL)
+    np.testing.assert_allclose(LSE, lse, atol=TOL)
+    np.testing.assert_allclose(dQ, gq, atol=TOL)
+    np.testing.assert_allclose(dK, gk, atol=TOL)
+    np.testing.assert_allclose(dV, gv, atol=TOL)
+    if not variant:
+        d2 = dense.bwd(Q, K, V, dO, S, T, head_past_mask=flags)
+        for a, b in zip((dQ, dK, dV), d2):
+            np.testing.assert_allclose(a, b, atol=TOL)
+
+
+# ---- closed form: zero keys => uniform attention over the visible set ---------------------------
+def test_zero_keys_closed_form_counts_the_context():
+    B, L, Hq, Hkv, d, S, T = 1, 120, 2, 2, 4, 40, 10
+    Q, K, V, _ = rand(B, L, Hq, Hkv, d)
+    K[:] = 0.0
+    O, LSE = oracle.fwd(Q, K, V, S, T, head_past_mask=[0, 1])
+    for p in range(L):
+        i, t = divmod(p, S)
+        n_local = t + 1 + (T if i > 0 else 0)          # S + M context of the cost model, Section 3.5
+        lo = p + 1 - n_local
+        assert abs(LSE[0, 0, p] - np.log(n_local)) < 1e-12
+        assert abs(LSE[0, 1, p] - np.log(p + 1)) < 1e-12
+        np.testing.assert_allclose(O[0, p, 0], V[0, lo:p + 1, 0].mean(axis=0), atol=1e-12)
+        np.testing.assert_allclose(O[0, p, 1], V[0, :p + 1, 1].mean(axis=0), atol=1e-12)
+
+
+def test_context_size_golden():
+    path = os.path.join(os.path.dirname(__file__), "golden", "context_size.txt")
+    rows = [tuple(int(x) for x in ln.split()) for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert rows
+    for S, M, i, t, n in rows:
+        L = (i + 1) * S
+        Q = np.zeros((1, L, 1, 1))
+        O, LSE = oracle.fwd(Q, Q, Q, S, M)
+        assert abs(np.exp(LSE[0, 0, i * S + t]) - n) < 1e-6
+
+
+# ---- finite differences with the stop-gradient semantics -----------------------------------------
+def fd_objective(Q, K, V, Kbar, Vbar, dO, S, T, flags):
+    """<O, dO> where every stop-gradient read takes its key/value from the constant copies
+    Kbar/Vbar (sg = identity forward, constant backward).  Built from oracle.fwd alone, one
+    segment at a time through its position offsets."""
+    L = Q.shape[1]
+    tot = 0.0
+    for i in range((L + S - 1) // S):
+        s0, s1 = i * S, min(L, (i + 1) * S)
+        a = max(0, s0 - T)
+        Km = np.concatenate([Kbar[:, :a], K[:, a:s1]], axis=1)
+        Vm = np.concatenate([Vbar[:, :a], V[:, a:s1]], axis=1)
+        O, _ = oracle.fwd(Q[:, s0:s1], Km, Vm, S, T, head_past_mask=flags, q_pos0=s0)
+        tot += float((O * dO[:, s0:s1]).sum())
+    return tot
+
+
+def test_gradients_match_central_finite_differences():
+    rng = np.random.default_rng(3)
+    B, L, Hq, Hkv, d, S, T = 1, 48, 2, 2, 4, 16, 5
+    flags = [1, 0]
+    Q, K, V, dO = rand(B, L, Hq, Hkv, d, rng)
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=flags)
+    eps = 1e-5
+    for name, X, G in (("Q", Q, dQ), ("K", K, dK), ("V", V, dV)):
+        idxs = [tuple(rng.integers(0, n) for n in X.shape) for _ in range(40)]
+        # make sure tail, non-tail and first-segment positions of both heads are probed
+        for pos in (0, S - T - 1, S - T, S - 1, S, 2 * S - 1, L - 1):
+            for hh in range(X.shape[2]):
+                idxs.append((0, pos, hh, int(rng.integers(0, d))))
+        for idx in idxs:
+            args = {"Q": Q, "K": K, "V": V}
+            Xp, Xm = X.copy(), X.copy()
+            Xp[idx] += eps
+            Xm[idx] -= eps
+            ap, am = dict(args), dict(args)
+            ap[name], am[name] = Xp, Xm
+            fp = fd_objective(ap["Q"], ap["K"], ap["V"], K, V, dO, S, T, flags)
+            fm = fd_objective(am["Q"], am["K"], am["V"], K, V, dO, S, T, flags)
+            fd = (fp - fm) / (2 * eps)
+            assert abs(fd - G[idx]) <= 1e-6 * max(1.0, abs(fd)), (name, idx, fd, G[idx])
+
+
+# ---- gradient reach: the tail is the only differentiable cross-segment state -------------------
+def test_loss_on_one_segment_reaches_only_that_segment_and_previous_tail():
+    B, L, Hq, Hkv, d, S, T = 1, 128, 4, 2, 8, 32, 8
+    Q, K, V, dO = rand(B, L, Hq, Hkv, d)
+    dO[:, :2 * S] = 0.0
+    dO[:, 3 * S:] = 0.0                      # loss on the third segment only
+    for flags in ([0, 0], [1, 0], [1, 1]):
+        dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=flags)
+        for G in (dK, dV):
+            assert np.all(G[:, :2 * S - T] == 0.0)       # exactly zero before the tail of segment 2
+            assert np.all(G[:, 3 * S:] == 0.0)
+            assert np.abs(G[:, 2 * S - T:3 * S]).min() > 0.0
+        assert np.all(dQ[:, :2 * S] == 0.0) and np.all(dQ[:, 3 * S:] == 0.0)
+
+
+def test_flag_changes_dq_but_not_the_reach_of_dk_dv():
+    B, L, Hq, Hkv, d, S, T = 1, 96, 2, 1, 8, 32, 8
+    Q, K, V, dO = rand(B, L, Hq, Hkv, d)
+    dQ0, dK0, dV0 = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=[0])
+    dQ1, dK1, dV1 = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=[1])
+    assert np.abs(dQ1[:, S:] - dQ0[:, S:]).max() > 1e-6          # sg keys do feed dQ
+    np.testing.assert_allclose(dQ1[:, :S], dQ0[:, :S], atol=TOL)  # first segment: nothing older to read
+    # a key outside the tail of segment 0 still gets nothing from segment 1 or 2 queries:
+    dO2 = dO.copy()
+    dO2[:, :S] = 0.0
+    _, dK2, dV2 = oracle.bwd(Q, K, V, dO2, S, T, head_past_mask=[1])
+    assert np.all(dK2[:, :S - T] == 0.0) and np.all(dV2[:, :S - T] == 0.0)
+
+
+def test_unflagged_output_ignores_keys_before_the_tail():
+    B, L, Hq, Hkv, d, S, T = 1, 96, 2, 2, 8, 32, 8
+    Q, K, V, _ = rand(B, L, Hq, Hkv, d)
+    O, LSE = oracle.fwd(Q, K, V, S, T, head_past_mask=[0, 1])
+    K2, V2 = K.copy(), V.copy()
+    K2[:, :2 * S - T] += 3.0
+    V2[:, :2 * S - T] -= 2.0
+    O2, LSE2 = oracle.fwd(Q, K2, V2, S, T, head_past_mask=[0, 1])
+    assert np.array_equal(O[:, 2 * S:, 0], O2[:, 2 * S:, 0]) and np.array_equal(LSE[:, 0, 2 * S:], LSE2[:, 0, 2 * S:])
+    assert np.abs(O[:, 2 * S:, 1] - O2[:, 2 * S:, 1]).max() > 1e-3   # the flagged head does read them
+
+
+# ---- cost model: pair counts --------------------------------------------------------------------
+@pytest.mark.parametrize("L,S,T", [(2048, 512, 128), (4096, 1024, 1024), (1536, 512, 0)])
+def test_pair_counts_match_closed_forms(L, S, T):
+    N = L // S
+    local = N * S * (S + 1) // 2 + (N - 1) * S * T
+    full = L * (L + 1) // 2
+    nv, nd = oracle.count_pairs(2, L, 4, 2, S, T, head_past_mask=[0, 1])
+    assert nv == 2 * 2 * (local + full) and nd == 2 * 4 * local
+    nv, nd = oracle.count_pairs(1, L, 4, 4, S, T)
+    assert nv == nd == 4 * local
+
+
+def test_benchmark_pair_counts():
+    # visible pairs of the benchmark configurations, recomputed from the closed forms
+    assert oracle.count_pairs(1, 2048, 4, 4, 512, 128)[0] == 2887680
+    nv, nd = oracle.count_pairs(2, 16384, 32, 8, 2048, 512, head_past_mask=[0, 0, 1, 0, 1, 0, 0, 0])
+    local = 8 * 2048 * 2049 // 2 + 7 * 2048 * 512
+    assert nv == 2 * (24 * local + 8 * (16384 * 16385 // 2)) == 3305635840
+    assert nd == 2 * 32 * local
+
+
+# ---- the two statements of the definition agree; streamed == one-shot ---------------------------
+def test_c_oracle_matches_dense_form_on_configuration_1():
+    import workloads
+    w = workloads.CONFIGS[0]
+    x = workloads.make_inputs(w)
+    Q, K, V, dO = (workloads.to_f64(x[k]) for k in ("Q", "K", "V", "dO"))
+    O, LSE = oracle.fwd(Q, K, V, w.S, w.T, x["mask"])
+    O2, LSE2 = dense.fwd(Q, K, V, w.S, w.T, x["mask"])
+    np.testing.assert_allclose(O, O2, atol=1e-12)
+    np.testing.assert_allclose(LSE, LSE2, atol=1e-12)
+    g1 = oracle.bwd(Q, K, V, dO, w.S, w.T, x["mask"])
+    g2 = dense.bwd(Q, K, V, dO, w.S, w.T, x["mask"])
+    for a, b in zip(g1, g2):
+        np.testing.assert_allclose(a, b, atol=1e-11)
+
+
+def test_streamed_segments_equal_one_shot_forward():
+    B, L, Hq, Hkv, d, S, T = 1, 128, 4, 2, 8, 32, 8
+    flags = [0, 1]
+    Q, K, V, _ = rand(B, L, Hq, Hkv, d)
+    O, LSE = oracle.fwd(Q, K, V, S, T, head_past_mask=flags)
+    for i in range(L // S):
+        s0, s1 = i * S, (i + 1) * S
+        # flagged head: whole history; the other head would need only [s0-T, s1) - pass that window
+        Oi, LSEi = oracle.fwd(Q[:, s0:s1], K[:, :s1], V[:, :s1], S, T, head_past_mask=flags, q_pos0=s0)
+        np.testing.assert_array_equal(Oi, O[:, s0:s1])
+        np.testing.assert_array_equal(LSEi, LSE[:, :, s0:s1])
+        a = max(0, s0 - T)
+        Ow, _ = oracle.fwd(Q[:, s0:s1, :2], K[:, a:s1, :1], V[:, a:s1, :1], S, T, q_pos0=s0, kv_pos0=a)
+        np.testing.assert_array_equal(Ow, O[:, s0:s1, :2])
+
+
+def test_invalid_configurations_are_rejected():
+    Q, K, V, _ = rand(1, 8, 2, 2, 4)
+    with pytest.raises(ValueError):
+        oracle.fwd(Q, K, V, 4, 5)          # tail longer than a segment
+    with pytest.raises(ValueError):
+        oracle.fwd(Q, K, V, 0, 0)
