@@ -1,0 +1,160 @@
+/*
+ * seg_attn.h - C ABI of the segment-level causal attention library for NVIDIA B200 (sm_100a).
+ *
+ * The operation (names follow the paper; its total length T is `L` here, its tail length M is `T`):
+ * a sequence of L positions is cut into non-overlapping segments of constant length S
+ * (Section 3.1 "Setup", Section 3.5).  Every head runs scaled dot-product attention
+ * softmax(Q K^T * sm_scale + mask) V (Appendix C, Eq. "attn") over a per-segment context
+ * (Appendix C, Eq. "ctx"):
+ *   - its own segment, causally (a query sees positions up to and including itself);
+ *   - the carried KV tail: the last T key/value positions of the immediately preceding
+ *     segment, the only differentiable cross-segment state (Section 3.4, "Local Continuity
+ *     Channel"); the first segment has no carried state (Section 3.1, C_0 empty);
+ *   - for KV heads flagged in `head_past_mask`, additionally every older key/value, read
+ *     forward-only: stop-gradient, no gradient reaches those K/V (Definition 3.2; Section 3.4,
+ *     "Long-Range Channel"; Appendix B, Lemma B.1).
+ * With global positions p (query) and j (key), i = p / S and a_i = max(0, i*S - T):
+ *     visible(p, j, c) <=> j <= p and (j >= a_i or head_past_mask[c] != 0)
+ *     diff(p, j)       <=> a_i <= j <= p            (reads that carry gradient into K/V)
+ * Query head h uses KV head c = h / (Hq / Hkv).
+ *
+ * Conventions that hold for every entry point unless it says otherwise:
+ *   - Tensor pointers are DEVICE pointers owned by the caller; the library never frees or
+ *     reallocates them.  Q, O, dO, dQ are bf16 [B][Lq][Hq][d]; K, V, dK, dV are bf16
+ *     [B][kv_len][Hkv][d]; addressing is by the element strides in seg_attn_params (the last
+ *     dimension is contiguous).  LSE is fp32, contiguous [B][Hq][Lq].
+ *   - `head_past_mask` is a HOST array of Hkv bytes (non-zero = flagged); it is read before
+ *     the call returns.
+ *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it; no entry point
+ *     synchronises the device except where stated.
+ *   - Errors are return codes.  Arguments are validated on the host before anything is
+ *     launched; on a non-zero return nothing was enqueued and the outputs are untouched.
+ *   - Base pointers must be 16-byte aligned and every stride a multiple of 8 elements
+ *     (tiles are moved by TMA).  d is 64 or 128.  0 <= T <= S.  Any Lq, kv_len >= 0.
+ *   - Arithmetic: bf16 inputs, fp32 accumulation on the tensor cores, fp32 softmax
+ *     statistics; P (and dS) are rounded to bf16 before the second product; outputs are
+ *     rounded to bf16 (round-to-nearest-even).  A query row with no visible key present
+ *     (possible only when kv_len does not reach it) yields O = 0, LSE = -inf.
+ */
+#ifndef SEG_ATTN_H_
+#define SEG_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SEGATTN_OK = 0,
+    SEGATTN_ERR_INVALID = 1,          /* bad shape, stride, alignment, null pointer, T > S, unsupported d */
+    SEGATTN_ERR_UNSUPPORTED_ARCH = 2, /* the current device is not compute capability 10.x */
+    SEGATTN_ERR_CUDA = 3,             /* a CUDA runtime/driver call failed; see seg_attn_last_cuda_error() */
+    SEGATTN_ERR_TIMEOUT = 4,          /* a bounded wait inside a kernel expired (see seg_attn_poll_status) */
+    SEGATTN_ERR_WORKSPACE = 5         /* workspace/state buffer missing, misaligned or too small */
+} segattn_status;
+
+typedef struct {
+    int32_t B;       /* batch */
+    int32_t Lq;      /* number of query rows per batch element */
+    int32_t kv_len;  /* number of key/value rows present per batch element */
+    int32_t Hq;      /* query heads */
+    int32_t Hkv;     /* key/value heads; Hq % Hkv == 0; at most 64 */
+    int32_t d;       /* head dimension: 64 or 128 */
+    int32_t S;       /* segment length, >= 1 */
+    int32_t T;       /* carried tail length, 0 <= T <= S */
+    int32_t q_pos0;  /* global position of query row 0 (0 for a whole sequence; i*S when streaming) */
+    int32_t kv_pos0; /* global position of key row 0 (may be negative: rows before position 0 are never visible) */
+    float sm_scale;  /* softmax scale; the paper uses 1/sqrt(d) */
+    int32_t reserved;
+    int64_t q_stride[3]; /* element strides of Q (and dQ) for (batch, position, head) */
+    int64_t k_stride[3]; /* element strides of K (and dK) */
+    int64_t v_stride[3]; /* element strides of V (and dV) */
+    int64_t o_stride[3]; /* element strides of O (and dO) */
+} seg_attn_params;
+
+/* Bytes of device scratch a call needs (is_bwd = 0: forward, none today; 1: backward, the
+ * fp32 row dots D[B][Hq][Lq], rounded up to 256).  Returns 0 for invalid params. */
+size_t seg_attn_workspace_bytes(const seg_attn_params* p, int is_bwd);
+
+/* Forward (Appendix C, Eqs. "attn" and "ctx"; mask as stated at the top of this file).
+ * O[b][r][h][:] = sum_j P_j V_j and LSE[b][h][r] = ln sum_j exp(sm_scale * <q,k_j>) over the
+ * visible j (natural logarithm of the scaled scores).  Fully overwrites O and LSE.
+ * `workspace` may be NULL (size 0). */
+segattn_status seg_attn_fwd(const seg_attn_params* p, const void* Q, const void* K, const void* V,
+                            const uint8_t* head_past_mask, void* O, float* LSE,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* Backward: the vector-Jacobian product of the forward for the cotangent dO (softmax VJP;
+ * stop-gradient per Definition 3.2 and Lemma B.1; the tail as sole differentiable
+ * cross-segment state per Section 3.4; one-transition reach of the K=1 discussion after
+ * Definition 3.2).  With P = exp(s - LSE), D = <dO,O>, dS = P * (dO V^T - D):
+ *   dQ_p = sm_scale * sum over visible j of dS_pj K_j          (stop-gradient keys included:
+ *                                                               sg cuts the K/V side only)
+ *   dK_j = sm_scale * sum over p with diff(p,j) of dS_pj Q_p,  dV_j = sum over the same p of P_pj dO_p
+ * summed over the query heads of the KV head.  A key position thus receives gradient only
+ * from queries of its own segment and, if it lies in the last T positions, of the next one.
+ * O and LSE must be the forward's results for the same inputs.  dQ, dK, dV are fully
+ * overwritten (no pre-zeroing).  `workspace` must hold seg_attn_workspace_bytes(p, 1) bytes,
+ * 256-byte aligned; it is scratch, dead after the enqueued work has run. */
+segattn_status seg_attn_bwd(const seg_attn_params* p, const void* Q, const void* K, const void* V,
+                            const void* O, const float* LSE, const void* dO,
+                            const uint8_t* head_past_mask, void* dQ, void* dK, void* dV,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- Streamed prefill: the segment recurrence (C_i, o_i) = F(x_i, C_{i-1}, R_{i-1}) of
+ * Definition 3.1 restricted to attention, with memory bounded as in Section 3.5 "Memory
+ * Complexity": flagged KV heads keep their whole key/value history (the append-only
+ * past-only pool of Section 3.4), the others keep only the T-position tail.
+ *
+ * The caller provides one device buffer for all persistent state.  In `p`, Lq is the
+ * segment length fed per step (must equal S), kv_len is the maximum total length the pool
+ * must hold, q_pos0/kv_pos0 are ignored, and the Q/O strides describe the per-step
+ * Q/O segment tensors [B][S][Hq][d], the K/V strides the per-step K/V segment tensors
+ * [B][S][Hkv][d].  The handle itself is a small host object (malloc'd by create, freed by
+ * destroy). */
+typedef struct seg_prefill_handle seg_prefill_handle;
+
+size_t seg_prefill_state_bytes(const seg_attn_params* p, const uint8_t* head_past_mask);
+segattn_status seg_prefill_create(const seg_attn_params* p, const uint8_t* head_past_mask,
+                                  void* state_mem, size_t state_bytes, seg_prefill_handle** out);
+/* Processes the next segment: appends its K/V to the retained state, writes O_seg
+ * [B][S][Hq][d] and LSE_seg [B][Hq][S] (the same values the whole-sequence forward gives for
+ * those rows), then rolls the tail.  Call once per segment, in order, on one stream. */
+segattn_status seg_prefill_step(seg_prefill_handle* h, const void* Qseg, const void* Kseg, const void* Vseg,
+                                void* Oseg, float* LSEseg, void* stream);
+segattn_status seg_prefill_reset(seg_prefill_handle* h); /* back to segment 0; state contents become dead */
+void seg_prefill_destroy(seg_prefill_handle* h);
+
+/* ---- Whole training-step call with HOST buffers (pinned or pageable): copies Q, K, V, dO to
+ * the device arena, runs forward and backward, copies O, LSE, dQ, dK, dV back, and
+ * synchronises `stream` before returning.  Host tensors are contiguous in the layouts
+ * above (strides in `p` are ignored).  dO_host == NULL runs the forward only (gradient
+ * outputs are then ignored).  `arena` is a caller-owned DEVICE buffer of at least
+ * seg_attn_host_arena_bytes(p) bytes, 256-byte aligned. */
+size_t seg_attn_host_arena_bytes(const seg_attn_params* p);
+segattn_status seg_attn_step_host(const seg_attn_params* p, const void* Q_host, const void* K_host,
+                                  const void* V_host, const void* dO_host, const uint8_t* head_past_mask,
+                                  void* O_host, float* LSE_host, void* dQ_host, void* dK_host, void* dV_host,
+                                  void* arena, size_t arena_bytes, void* stream);
+
+/* ---- Status and accounting */
+/* Synchronises `stream`, then reads and clears the device status word that kernels set when a
+ * bounded wait expires.  Returns SEGATTN_OK, SEGATTN_ERR_TIMEOUT or SEGATTN_ERR_CUDA. */
+segattn_status seg_attn_poll_status(void* stream);
+const char* seg_attn_status_string(segattn_status s);
+/* Last CUDA error code (cudaError_t or CUresult as int) recorded by this thread's failing call. */
+int seg_attn_last_cuda_error(void);
+/* Exact (query,key) pair counts of the mask summed over batch and query heads (the cost
+ * model of Section 3.5 evaluated element-exactly), and the number of 128x128 tiles the
+ * forward kernel visits.  Any of the output pointers may be NULL. */
+segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* head_past_mask,
+                                    int64_t* pairs_visible, int64_t* pairs_diff, int64_t* fwd_tiles);
+/* Number of kernel launches the library has enqueued so far in this process. */
+int64_t seg_attn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEG_ATTN_H_ */

@@ -1,0 +1,10 @@
+"""B200-native segment-level causal attention: thin Python binding over the C-ABI library.
+
+Every step of the path runs in the CUDA kernels of ``libsegattn.so``; this package only
+marshals arguments.  PyTorch supplies device memory and streams.
+"""
+from .binding import (SegAttnError, Prefill, count_pairs, launch_count, lib, params_for, poll_status,
+                      seg_attn_bwd, seg_attn_fwd, seg_attn_step_host, workspace_bytes)
+
+__all__ = ["SegAttnError", "Prefill", "count_pairs", "launch_count", "lib", "params_for", "poll_status",
+           "seg_attn_bwd", "seg_attn_fwd", "seg_attn_step_host", "workspace_bytes"]

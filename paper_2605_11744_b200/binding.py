@@ -1,0 +1,243 @@
+"""ctypes binding with the same names as the C ABI in ``include/seg_attn.h``.
+
+Argument marshalling only: pointers, strides and the stream are taken from torch tensors and
+handed to the library.  There is no fallback: if ``libsegattn.so`` is missing the import fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libsegattn.so")
+
+
+class SegAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().seg_attn_status_string(status).decode()
+        extra = " (cuda/driver code %d)" % lib().seg_attn_last_cuda_error() if status in (3, 4) else ""
+        super().__init__("%s: %s%s" % (where, msg, extra))
+
+
+class Params(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("B", "Lq", "kv_len", "Hq", "Hkv", "d", "S", "T", "q_pos0", "kv_pos0")] + \
+               [("sm_scale", ctypes.c_float), ("reserved", ctypes.c_int32),
+                ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
+                ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it has not been built (no CPU or eager fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError("libsegattn.so is not built: run `python -m paper_2605_11744_b200.build` "
+                              "(or __graft_entry__.build()); there is no fallback path")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, u8p, fp = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+        pp = ctypes.POINTER(Params)
+        L.seg_attn_workspace_bytes.restype = ctypes.c_size_t
+        L.seg_attn_workspace_bytes.argtypes = [pp, ctypes.c_int]
+        L.seg_attn_fwd.argtypes = [pp, vp, vp, vp, u8p, vp, fp, vp, ctypes.c_size_t, vp]
+        L.seg_attn_bwd.argtypes = [pp, vp, vp, vp, vp, fp, vp, u8p, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.seg_prefill_state_bytes.restype = ctypes.c_size_t
+        L.seg_prefill_state_bytes.argtypes = [pp, u8p]
+        L.seg_prefill_create.argtypes = [pp, u8p, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+        L.seg_prefill_step.argtypes = [vp, vp, vp, vp, vp, fp, vp]
+        L.seg_prefill_reset.argtypes = [vp]
+        L.seg_prefill_destroy.argtypes = [vp]
+        L.seg_prefill_destroy.restype = None
+        L.seg_attn_host_arena_bytes.restype = ctypes.c_size_t
+        L.seg_attn_host_arena_bytes.argtypes = [pp]
+        L.seg_attn_step_host.argtypes = [pp, vp, vp, vp, vp, u8p, vp, fp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.seg_attn_poll_status.argtypes = [vp]
+        L.seg_attn_status_string.restype = ctypes.c_char_p
+        L.seg_attn_status_string.argtypes = [ctypes.c_int]
+        L.seg_attn_last_cuda_error.restype = ctypes.c_int
+        L.seg_attn_launch_count.restype = ctypes.c_int64
+        L.seg_attn_count_pairs.argtypes = [pp, u8p] + [ctypes.POINTER(ctypes.c_int64)] * 3
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise SegAttnError(status, where)
+
+
+def _mask_arr(head_past_mask, Hkv: int) -> np.ndarray:
+    m = np.zeros(Hkv, dtype=np.uint8) if head_past_mask is None else \
+        np.ascontiguousarray(np.asarray(head_past_mask) != 0, dtype=np.uint8)
+    if m.shape != (Hkv,):
+        raise ValueError("head_past_mask must have Hkv entries")
+    return m
+
+
+def _strides3(t: torch.Tensor):
+    if t.dim() != 4 or (t.shape[3] > 1 and t.stride(3) != 1):
+        raise ValueError("expected a [B, L, H, d] tensor with a contiguous last dimension")
+    return (ctypes.c_int64 * 3)(t.stride(0), t.stride(1), t.stride(2))
+
+
+def params_for(Q, K, V, O, S: int, T: int, sm_scale: Optional[float] = None, q_pos0: int = 0,
+               kv_pos0: int = 0) -> Params:
+    """seg_attn_params for [B, L, H, d] tensors (only shapes and strides are read)."""
+    B, Lq, Hq, d = Q.shape
+    kv_len, Hkv = K.shape[1], K.shape[2]
+    p = Params()
+    p.B, p.Lq, p.kv_len, p.Hq, p.Hkv, p.d = B, Lq, kv_len, Hq, Hkv, d
+    p.S, p.T, p.q_pos0, p.kv_pos0 = S, T, q_pos0, kv_pos0
+    p.sm_scale = float(sm_scale if sm_scale is not None else d ** -0.5)
+    p.q_stride, p.k_stride, p.v_stride, p.o_stride = _strides3(Q), _strides3(K), _strides3(V), _strides3(O)
+    return p
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None or t.numel() == 0 else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _need_cuda_bf16(*ts):
+    for t in ts:
+        if t.device.type != "cuda" or t.dtype != torch.bfloat16:
+            raise ValueError("tensors must be bf16 CUDA tensors")
+
+
+def workspace_bytes(p: Params, is_bwd: bool) -> int:
+    return int(lib().seg_attn_workspace_bytes(ctypes.byref(p), int(is_bwd)))
+
+
+def seg_attn_fwd(Q, K, V, S: int, T: int, head_past_mask=None, sm_scale=None, q_pos0=0, kv_pos0=0,
+                 out=None, lse=None, stream=None):
+    """O [B,Lq,Hq,d] bf16 and LSE [B,Hq,Lq] fp32 (natural log) - one call of the C entry point `seg_attn_fwd`."""
+    _need_cuda_bf16(Q, K, V)
+    O = torch.empty_like(Q) if out is None else out
+    LSE = torch.empty((Q.shape[0], Q.shape[2], Q.shape[1]), dtype=torch.float32, device=Q.device) if lse is None else lse
+    p = params_for(Q, K, V, O, S, T, sm_scale, q_pos0, kv_pos0)
+    m = _mask_arr(head_past_mask, p.Hkv)
+    _check(lib().seg_attn_fwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), m.ctypes.data, _ptr(O), _ptr(LSE),
+                              None, 0, _stream(stream)), "seg_attn_fwd")
+    return O, LSE
+
+
+def seg_attn_bwd(Q, K, V, O, LSE, dO, S: int, T: int, head_past_mask=None, sm_scale=None, q_pos0=0, kv_pos0=0,
+                 workspace: Optional[torch.Tensor] = None, stream=None):
+    """dQ, dK, dV (bf16) - one call of the C entry point `seg_attn_bwd`."""
+    _need_cuda_bf16(Q, K, V, O, dO)
+    if dO.stride() != O.stride():
+        raise ValueError("dO must have the strides of O")
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    if dQ.stride() != Q.stride() or dK.stride() != K.stride() or dV.stride() != V.stride():
+        raise ValueError("Q, K, V must be dense (non-overlapping) tensors")
+    p = params_for(Q, K, V, O, S, T, sm_scale, q_pos0, kv_pos0)
+    m = _mask_arr(head_past_mask, p.Hkv)
+    need = workspace_bytes(p, True)
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device) if workspace is None else workspace
+    _check(lib().seg_attn_bwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), _ptr(dO),
+                              m.ctypes.data, _ptr(dQ), _ptr(dK), _ptr(dV), ctypes.c_void_p(ws.data_ptr()),
+                              ws.numel(), _stream(stream)), "seg_attn_bwd")
+    return dQ, dK, dV
+
+
+def seg_attn_step_host(Q, K, V, dO, S: int, T: int, head_past_mask=None, sm_scale=None,
+                       arena: Optional[torch.Tensor] = None, outs=None, stream=None):
+    """Forward (+ backward if dO is given) with HOST bf16 tensors in, HOST tensors out, through the
+    C entry point `seg_attn_step_host`; copies both ways happen inside the call."""
+    for t in (Q, K, V) + ((dO,) if dO is not None else ()):
+        if t.device.type != "cpu" or t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("host entry point takes contiguous bf16 CPU tensors")
+    p = params_for(Q, K, V, Q, S, T, sm_scale)
+    m = _mask_arr(head_past_mask, p.Hkv)
+    need = int(lib().seg_attn_host_arena_bytes(ctypes.byref(p)))
+    if arena is None:
+        arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+    if outs is None:
+        pin = torch.cuda.is_available()
+        mk = lambda like: torch.empty(like.shape, dtype=like.dtype, pin_memory=pin)
+        outs = {"O": mk(Q), "LSE": torch.empty((p.B, p.Hq, p.Lq), dtype=torch.float32, pin_memory=pin)}
+        if dO is not None:
+            outs.update(dQ=mk(Q), dK=mk(K), dV=mk(V))
+    g = lambda k: _ptr(outs.get(k))
+    _check(lib().seg_attn_step_host(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO), m.ctypes.data,
+                                    g("O"), g("LSE"), g("dQ"), g("dK"), g("dV"),
+                                    ctypes.c_void_p(arena.data_ptr()), arena.numel(), _stream(stream)),
+           "seg_attn_step_host")
+    return outs
+
+
+class Prefill:
+    """Streamed, memory-bounded prefill: wraps seg_prefill_create/step/reset/destroy.  The persistent
+    state (the flagged heads' key/value pool and the other heads' tail) lives in one torch buffer."""
+
+    def __init__(self, B, S, T, Hq, Hkv, d, max_len, head_past_mask=None, sm_scale=None, device="cuda"):
+        p = Params()
+        p.B, p.Lq, p.kv_len, p.Hq, p.Hkv, p.d, p.S, p.T = B, S, max_len, Hq, Hkv, d, S, T
+        p.sm_scale = float(sm_scale if sm_scale is not None else d ** -0.5)
+        p.q_stride = p.o_stride = (ctypes.c_int64 * 3)(S * Hq * d, Hq * d, d)
+        p.k_stride = p.v_stride = (ctypes.c_int64 * 3)(S * Hkv * d, Hkv * d, d)
+        self.params = p
+        self.mask = _mask_arr(head_past_mask, Hkv)
+        self.state_bytes = int(lib().seg_prefill_state_bytes(ctypes.byref(p), self.mask.ctypes.data))
+        self.state = torch.empty(max(self.state_bytes, 256), dtype=torch.uint8, device=device)
+        h = ctypes.c_void_p()
+        _check(lib().seg_prefill_create(ctypes.byref(p), self.mask.ctypes.data, ctypes.c_void_p(self.state.data_ptr()),
+                                        self.state.numel(), ctypes.byref(h)), "seg_prefill_create")
+        self._h = h
+
+    def step(self, Qseg, Kseg, Vseg, out=None, lse=None, stream=None):
+        _need_cuda_bf16(Qseg, Kseg, Vseg)
+        p = self.params
+        if tuple(Qseg.shape) != (p.B, p.S, p.Hq, p.d) or tuple(Kseg.shape) != (p.B, p.S, p.Hkv, p.d) or \
+                Kseg.shape != Vseg.shape or not (Qseg.is_contiguous() and Kseg.is_contiguous() and Vseg.is_contiguous()):
+            raise ValueError("segment tensors must be contiguous [B,S,H,d]")
+        O = torch.empty_like(Qseg) if out is None else out
+        LSE = torch.empty((p.B, p.Hq, p.S), dtype=torch.float32, device=Qseg.device) if lse is None else lse
+        _check(lib().seg_prefill_step(self._h, _ptr(Qseg), _ptr(Kseg), _ptr(Vseg), _ptr(O), _ptr(LSE),
+                                      _stream(stream)), "seg_prefill_step")
+        return O, LSE
+
+    def reset(self):
+        _check(lib().seg_prefill_reset(self._h), "seg_prefill_reset")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().seg_prefill_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def poll_status(stream=None):
+    _check(lib().seg_attn_poll_status(_stream(stream)), "seg_attn_poll_status")
+
+
+def launch_count() -> int:
+    return int(lib().seg_attn_launch_count())
+
+
+def count_pairs(B, Lq, Hq, Hkv, d, S, T, head_past_mask=None, kv_len=None, q_pos0=0, kv_pos0=0):
+    """(visible pairs, differentiable pairs, 128x128 forward tiles visited), summed over batch and query heads."""
+    p = Params()
+    p.B, p.Lq, p.kv_len, p.Hq, p.Hkv, p.d, p.S, p.T = B, Lq, Lq if kv_len is None else kv_len, Hq, Hkv, d, S, T
+    p.q_pos0, p.kv_pos0, p.sm_scale = q_pos0, kv_pos0, 1.0
+    m = _mask_arr(head_past_mask, Hkv)
+    a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    _check(lib().seg_attn_count_pairs(ctypes.byref(p), m.ctypes.data, ctypes.byref(a), ctypes.byref(b),
+                                      ctypes.byref(c)), "seg_attn_count_pairs")
+    return a.value, b.value, c.value

@@ -1,0 +1,107 @@
+// Segment / tail / past-access mask arithmetic shared by the host-side scheduler and the
+// kernels, and the parameter blocks the kernels take.
+//
+// Global positions: query row r is position p = q_pos0 + r, key row jl is position
+// j = kv_pos0 + jl.  With i = p / S and a_i = max(0, i*S - T) (start of the carried tail of
+// the previous segment, Section 3.4 "Local Continuity Channel"; C_0 empty, Section 3.1):
+//   visible(p, j) <=> lo_vis(p) <= j <= p,  lo_vis(p) = flagged ? 0 : a_i   (Appendix C, Eq. "ctx")
+//   diff(p, j)    <=> a_i <= j <= p     (reads whose K/V receive gradient; Definition 3.2)
+// For a fixed key j the differentiable queries are also one interval: p in [j, hi_diff(j)),
+// hi_diff(j) = end of j's segment, plus the whole next segment when j lies in the last T
+// positions of its segment.
+#pragma once
+#include <cstdint>
+#include <cuda.h>
+
+namespace segattn {
+
+constexpr int kTile = 128;     // query rows per tile = key rows per tile
+constexpr int kMaxKvHeads = 64;
+
+struct MaskGeom {
+    int S, T;
+    int q_pos0, kv_pos0;
+    int Lq, kv_len;
+};
+
+__host__ __device__ inline long long tail_start(const MaskGeom& g, long long p) {
+    long long a = (p / g.S) * (long long)g.S - g.T;
+    return a < 0 ? 0 : a;
+}
+__host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, bool flagged) {
+    return flagged ? 0 : tail_start(g, p);
+}
+// one past the last query position that differentiably reads key position j
+__host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j) {
+    long long seg_end = (j / g.S + 1) * (long long)g.S;
+    return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
+}
+
+// Local key-row range [jl_lo, jl_hi] (inclusive) that the query tile starting at row r0 can see;
+// empty when jl_hi < jl_lo.
+__host__ __device__ inline void q_tile_kv_range(const MaskGeom& g, int r0, bool flagged, bool diff_only,
+                                                long long* jl_lo, long long* jl_hi) {
+    int r_last = r0 + kTile - 1;
+    if (r_last > g.Lq - 1) r_last = g.Lq - 1;
+    long long p0 = (long long)g.q_pos0 + r0, p1 = (long long)g.q_pos0 + r_last;
+    long long lo = diff_only ? tail_start(g, p0) : lo_visible(g, p0, flagged);
+    long long a = lo - g.kv_pos0, b = p1 - g.kv_pos0;
+    if (a < 0) a = 0;
+    if (b > g.kv_len - 1) b = g.kv_len - 1;
+    *jl_lo = a;
+    *jl_hi = b;
+}
+// Query-row range [r_lo, r_hi] (inclusive) that differentiably reads some key of the key tile
+// starting at local row c0; empty when r_hi < r_lo.
+__host__ __device__ inline void kv_tile_q_range(const MaskGeom& g, int c0, long long* r_lo, long long* r_hi) {
+    int c_last = c0 + kTile - 1;
+    if (c_last > g.kv_len - 1) c_last = g.kv_len - 1;
+    long long j0 = (long long)g.kv_pos0 + c0, j1 = (long long)g.kv_pos0 + c_last;
+    if (j1 < 0) { *r_lo = 0; *r_hi = -1; return; }
+    if (j0 < 0) j0 = 0;
+    long long a = j0 - g.q_pos0;              // first query position is the key itself
+    long long b = hi_diff(g, j1) - 1 - g.q_pos0;  // hi_diff is non-decreasing in j
+    if (a < 0) a = 0;
+    if (b > g.Lq - 1) b = g.Lq - 1;
+    *r_lo = a;
+    *r_hi = b;
+}
+
+// Which KV "slot" (head index inside the K/V tensors handed to the kernel) serves which
+// logical KV head, in what launch order, and whether it is flagged.
+struct HeadTable {
+    uint8_t order[kMaxKvHeads];    // slots sorted flagged-first (heaviest work first)
+    uint8_t flag[kMaxKvHeads];     // per slot
+    uint8_t logical[kMaxKvHeads];  // per slot: logical KV head (query heads logical*g .. +g-1)
+    int n_slots, n_flagged;
+};
+
+struct alignas(64) FwdParams {
+    CUtensorMap tq, tk, tv;  // bf16 (d, heads, rows, batch), box (64, 1, 128, 1), 128-byte swizzle
+    void* O;
+    float* LSE;
+    long long o_stride[3];
+    MaskGeom geom;
+    int B, Hq, g;
+    int n_qtiles;
+    float scale_log2;  // sm_scale * log2(e)
+    HeadTable heads;
+};
+
+struct alignas(64) BwdParams {
+    CUtensorMap tq, tk, tv, tdo;  // same form as above
+    const float* LSE;             // [B][Hq][Lq]
+    const float* Dvec;            // [B][Hq][Lq]  row dots <dO, O>
+    void* dQ;
+    void* dK;
+    void* dV;
+    long long q_stride[3], k_stride[3], v_stride[3];
+    MaskGeom geom;
+    int B, Hq, Hkv, g;
+    int n_qtiles, n_kvtiles;
+    float scale_log2;  // sm_scale * log2(e)
+    float sm_scale;
+    HeadTable heads;
+};
+
+}  // namespace segattn
