@@ -165,10 +165,14 @@ int oracle_seg_attn_bwd(const oracle_cfg *c, const double *Q, const double *K, c
     if (!cfg_ok(c)) return 1;
     const int g = c->Hq / c->Hkv, d = c->d;
     const long kstride = (long)c->Hkv * d;
-    memset(dK, 0, sizeof(double) * (size_t)c->B * c->Lk * c->Hkv * d);
-    memset(dV, 0, sizeof(double) * (size_t)c->B * c->Lk * c->Hkv * d);
+    const long nrows = (long)c->B * c->Hq * c->Lq;
     int fail = 0;
-    const long nunits = (long)c->B * c->Hkv; /* one unit owns dK/dV of one (batch, KV head) */
+    /* per query row: LSE_p and D_p = <dO_p, O_p>, kept for the key-side sums below */
+    double *LSE = (double *)malloc(sizeof(double) * (size_t)(nrows > 0 ? nrows : 1));
+    double *Dv = (double *)malloc(sizeof(double) * (size_t)(nrows > 0 ? nrows : 1));
+    if (!LSE || !Dv) { free(LSE); free(Dv); return 2; }
+
+    /* Query side, one row at a time: dQ_p = scale * sum over visible j of dS_j k_j. */
 #pragma omp parallel
     {
         double *pbuf = (double *)malloc(sizeof(double) * (size_t)(c->Lk > 0 ? c->Lk : 1));
@@ -177,52 +181,83 @@ int oracle_seg_attn_bwd(const oracle_cfg *c, const double *Q, const double *K, c
 #pragma omp atomic write
             fail = 1;
         }
-#pragma omp for schedule(dynamic, 1)
-        for (long u = 0; u < nunits; ++u) {
+#pragma omp for schedule(dynamic, 16)
+        for (long idx = 0; idx < nrows; ++idx) {
             if (!pbuf || !orow) continue;
-            int b = (int)(u / c->Hkv), kvh = (int)(u % c->Hkv);
-            int flag = head_past_mask[kvh] != 0;
+            long r = idx % c->Lq;
+            int h = (int)((idx / c->Lq) % c->Hq);
+            int b = (int)(idx / ((long)c->Lq * c->Hq));
+            int kvh = h / g;
+            long p = (long)c->q_pos0 + r, lo_vis, lo_diff, j0, j1;
+            row_bounds(c, head_past_mask[kvh] != 0, p, &lo_vis, &lo_diff);
+            local_range(c, lo_vis, p, &j0, &j1);
             const double *Kb = K + (long)b * c->Lk * c->Hkv * d;
             const double *Vb = V + (long)b * c->Lk * c->Hkv * d;
-            double *dKb = dK + (long)b * c->Lk * c->Hkv * d;
-            double *dVb = dV + (long)b * c->Lk * c->Hkv * d;
-            for (int h = kvh * g; h < (kvh + 1) * g; ++h) {
-                for (long r = 0; r < c->Lq; ++r) {
-                    long p = (long)c->q_pos0 + r, lo_vis, lo_diff, j0, j1, jd0, jd1;
-                    row_bounds(c, flag, p, &lo_vis, &lo_diff);
-                    local_range(c, lo_vis, p, &j0, &j1);
-                    local_range(c, lo_diff, p, &jd0, &jd1);
-                    const long qoff = (((long)b * c->Lq + r) * c->Hq + h) * d;
-                    const double *q = Q + qoff, *go = dO + qoff;
-                    double *gq = dQ + qoff;
-                    for (int e = 0; e < d; ++e) gq[e] = 0.0;
-                    if (j1 <= j0) continue;
-                    row_forward(c, q, Kb, Vb, kvh, j0, j1, pbuf, orow);
-                    double D = 0.0;
-                    for (int e = 0; e < d; ++e) D += go[e] * orow[e];
-                    for (long jl = j0; jl < j1; ++jl) {
-                        const double *k = Kb + jl * kstride + (long)kvh * d;
-                        const double *v = Vb + jl * kstride + (long)kvh * d;
-                        double dP = 0.0;
-                        for (int e = 0; e < d; ++e) dP += go[e] * v[e];
-                        double P = pbuf[jl];
-                        double dS = P * (dP - D);
-                        for (int e = 0; e < d; ++e) gq[e] += c->scale * dS * k[e];
-                        if (jl >= jd0 && jl < jd1) { /* differentiable read: own segment or tail */
-                            double *gk = dKb + jl * kstride + (long)kvh * d;
-                            double *gv = dVb + jl * kstride + (long)kvh * d;
-                            for (int e = 0; e < d; ++e) {
-                                gk[e] += c->scale * dS * q[e];
-                                gv[e] += P * go[e];
-                            }
-                        }
-                    }
-                }
+            const long qoff = (((long)b * c->Lq + r) * c->Hq + h) * d;
+            const double *q = Q + qoff, *go = dO + qoff;
+            double *gq = dQ + qoff;
+            for (int e = 0; e < d; ++e) gq[e] = 0.0;
+            const long sidx = ((long)b * c->Hq + h) * c->Lq + r;
+            LSE[sidx] = -INFINITY;
+            Dv[sidx] = 0.0;
+            if (j1 <= j0) continue;
+            LSE[sidx] = row_forward(c, q, Kb, Vb, kvh, j0, j1, pbuf, orow);
+            double D = 0.0;
+            for (int e = 0; e < d; ++e) D += go[e] * orow[e];
+            Dv[sidx] = D;
+            for (long jl = j0; jl < j1; ++jl) {
+                const double *k = Kb + jl * kstride + (long)kvh * d;
+                const double *v = Vb + jl * kstride + (long)kvh * d;
+                double dP = 0.0;
+                for (int e = 0; e < d; ++e) dP += go[e] * v[e];
+                double dS = pbuf[jl] * (dP - D);
+                for (int e = 0; e < d; ++e) gq[e] += c->scale * dS * k[e];
             }
         }
         free(pbuf);
         free(orow);
     }
+
+    /* Key side, one key row at a time: sums over the query heads of the group and over the
+     * query rows whose read of this key is differentiable (own segment or carried tail);
+     * stop-gradient reads contribute nothing. */
+    const long nkeys = (long)c->B * c->Lk * c->Hkv;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (long idx = 0; idx < nkeys; ++idx) {
+        int kvh = (int)(idx % c->Hkv);
+        long jl = (idx / c->Hkv) % c->Lk;
+        int b = (int)(idx / ((long)c->Hkv * c->Lk));
+        long j = (long)c->kv_pos0 + jl;
+        int flag = head_past_mask[kvh] != 0;
+        const double *k = K + (((long)b * c->Lk + jl) * c->Hkv + kvh) * d;
+        const double *v = V + (((long)b * c->Lk + jl) * c->Hkv + kvh) * d;
+        double *gk = dK + (((long)b * c->Lk + jl) * c->Hkv + kvh) * d;
+        double *gv = dV + (((long)b * c->Lk + jl) * c->Hkv + kvh) * d;
+        for (int e = 0; e < d; ++e) { gk[e] = 0.0; gv[e] = 0.0; }
+        if (j < 0) continue;
+        for (int h = kvh * g; h < (kvh + 1) * g; ++h) {
+            long r_first = j - c->q_pos0;                 /* causal: only rows at or after the key */
+            if (r_first < 0) r_first = 0;
+            for (long r = r_first; r < c->Lq; ++r) {
+                long p = (long)c->q_pos0 + r, lo_vis, lo_diff;
+                row_bounds(c, flag, p, &lo_vis, &lo_diff);
+                if (j < lo_diff) continue;                /* not visible, or a stop-gradient read */
+                const long qoff = (((long)b * c->Lq + r) * c->Hq + h) * d;
+                const double *q = Q + qoff, *go = dO + qoff;
+                const long sidx = ((long)b * c->Hq + h) * c->Lq + r;
+                double s = 0.0, dP = 0.0;
+                for (int e = 0; e < d; ++e) { s += q[e] * k[e]; dP += go[e] * v[e]; }
+                double P = exp(s * c->scale - LSE[sidx]);
+                double dS = P * (dP - Dv[sidx]);
+                for (int e = 0; e < d; ++e) {
+                    gk[e] += c->scale * dS * q[e];
+                    gv[e] += P * go[e];
+                }
+            }
+        }
+    }
+    free(LSE);
+    free(Dv);
     return fail ? 2 : 0;
 }
 

@@ -1,2 +1,60 @@
+// Data movement of the streamed prefill (the segment recurrence of Definition 3.1): append one
+// segment's K/V to the retained state, and carry the last T positions over as the next tail
+// (Section 3.4: past-only pool for flagged heads, carried KV tail for the others).
 #pragma once
-#include "mask.cuh"
+#include <cstdint>
+#include <cuda_bf16.h>
+
+namespace segattn {
+
+struct PrefillCopyParams {
+    const uint4* Kseg;  // [B][S][Hkv][d] (strides in 16-byte units below)
+    const uint4* Vseg;
+    uint4* Kpool;       // [B][n_flag][Lmax][d]
+    uint4* Vpool;
+    uint4* Kwin;        // [B][n_unflag][T+S][d]: rows [0,T) previous tail, rows [T,T+S) current segment
+    uint4* Vwin;
+    long long seg_stride[3];  // (batch, position, head) of Kseg/Vseg, in uint4 units
+    int B, S, T, Hkv, Lmax, n_flag, n_unflag;
+    int d16;            // d * 2 / 16: uint4 per head row
+    int pos0;           // first global position of this segment
+    uint8_t slot_of_head[64];  // KV head -> slot inside its class (pool slot or window slot)
+    uint8_t flag_of_head[64];
+};
+
+// one thread per 16 bytes of the incoming segment (K and V both)
+__global__ void __launch_bounds__(256) prefill_append_kernel(const PrefillCopyParams prm) {
+    const long long n = (long long)prm.B * prm.S * prm.Hkv * prm.d16;
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= n) return;
+    const int e = (int)(idx % prm.d16);
+    const int h = (int)((idx / prm.d16) % prm.Hkv);
+    const int r = (int)((idx / ((long long)prm.d16 * prm.Hkv)) % prm.S);
+    const int b = (int)(idx / ((long long)prm.d16 * prm.Hkv * prm.S));
+    const long long src = b * prm.seg_stride[0] + (long long)r * prm.seg_stride[1] + h * prm.seg_stride[2] + e;
+    const uint4 k = prm.Kseg[src], v = prm.Vseg[src];
+    const int slot = prm.slot_of_head[h];
+    if (prm.flag_of_head[h]) {
+        const long long dst = (((long long)b * prm.n_flag + slot) * prm.Lmax + prm.pos0 + r) * prm.d16 + e;
+        prm.Kpool[dst] = k;
+        prm.Vpool[dst] = v;
+    } else {
+        const long long dst = (((long long)b * prm.n_unflag + slot) * (prm.T + prm.S) + prm.T + r) * prm.d16 + e;
+        prm.Kwin[dst] = k;
+        prm.Vwin[dst] = v;
+    }
+}
+
+// window rows [S, S+T) (the last T positions of the segment just processed) -> rows [0, T)
+__global__ void __launch_bounds__(256) prefill_roll_tail_kernel(uint4* Kwin, uint4* Vwin, int n_units, int S, int T,
+                                                                int d16) {
+    const long long per = (long long)T * d16;
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= per * n_units) return;
+    const long long u = idx / per, off = idx % per;
+    const long long base = u * (long long)(T + S) * d16;
+    Kwin[base + off] = Kwin[base + (long long)S * d16 + off];
+    Vwin[base + off] = Vwin[base + (long long)S * d16 + off];
+}
+
+}  // namespace segattn
