@@ -184,7 +184,10 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
         if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
 
         const float sl2 = prm.scale_log2;
-        float m_run = -INFINITY, l_run = 0.f;
+        // l_run: row sum of the unrounded p (gives LSE); lr_run: row sum of the bf16-rounded p that
+        // the PV product actually uses, so that O = sum(p~ v) / sum(p~) stays a convex combination
+        // of value rows even when one key dominates (outlier keys)
+        float m_run = -INFINITY, l_run = 0.f, lr_run = 0.f;
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int c0 = (t_lo + j) * kTile;
@@ -218,6 +221,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
             if (grow) {
                 alpha = ex2(m_run - m_new);  // 0 when nothing was accumulated yet
                 l_run *= alpha;
+                lr_run *= alpha;
                 m_run = m_new;
             }
             if (j > 0 && __any_sync(0xffffffffu, grow)) {
@@ -234,7 +238,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
             }
             // pass 2: p = 2^(s*scale*log2e - m); row sum from the unrounded p; P to TMEM as bf16
             const float m_eff = (m_run == -INFINITY) ? 0.f : m_run;
-            float lsum = 0.f;
+            float lsum = 0.f, lsum_r = 0.f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t v[32];
@@ -251,11 +255,14 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
                         if (!(col + 1 >= vlo && col + 1 <= vhi)) p1 = 0.f;
                     }
                     lsum += p0 + p1;
-                    pk[i / 2] = pack_bf16(p0, p1);
+                    const uint32_t pr = pack_bf16(p0, p1);
+                    lsum_r += __uint_as_float(pr << 16) + __uint_as_float(pr & 0xffff0000u);
+                    pk[i / 2] = pr;
                 }
                 tmem_st_x16(tP + lane_off + c * 16, pk);
             }
             l_run += lsum;
+            lr_run += lsum_r;
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(kBarPFull));
@@ -263,8 +270,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
         // ---------------- epilogue ----------------
         if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), 0, 9));
         tc_fence_after();
-        const bool have = n_tiles > 0 && ok && l_run > 0.f;
-        const float inv_l = have ? 1.f / l_run : 0.f;
+        const bool have = n_tiles > 0 && ok && l_run > 0.f && lr_run > 0.f;
+        const float inv_l = have ? 1.f / lr_run : 0.f;
         if (r < geo.Lq && (ok || n_tiles == 0)) {
             __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(prm.O) + it.b * prm.o_stride[0] +
                                   (long long)r * prm.o_stride[1] + it.hq * prm.o_stride[2];

@@ -1,0 +1,126 @@
+"""CPU-side checks of the boundary: the library loads without a GPU, exports every symbol the
+header declares, validates arguments before touching a device, and its pair counter agrees
+with the oracle's enumeration of the mask."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+import paper_2605_11744_b200 as sa
+from paper_2605_11744_b200.binding import Params
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "seg_attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(seg_(?:attn|prefill)_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert "seg_attn_fwd" in names and "seg_attn_bwd" in names and "seg_prefill_step" in names
+    L = sa.lib()
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_status_strings():
+    L = sa.lib()
+    assert L.seg_attn_status_string(0) == b"ok"
+    for s in range(1, 6):
+        assert len(L.seg_attn_status_string(s)) > 3
+
+
+def _params(**kw):
+    p = Params()
+    base = dict(B=1, Lq=256, kv_len=256, Hq=4, Hkv=2, d=128, S=64, T=16, q_pos0=0, kv_pos0=0, sm_scale=0.1)
+    base.update(kw)
+    for k, v in base.items():
+        setattr(p, k, v)
+    for name, H in (("q_stride", base["Hq"]), ("o_stride", base["Hq"]), ("k_stride", base["Hkv"]), ("v_stride", base["Hkv"])):
+        L = base["Lq"] if name[0] in "qo" else base["kv_len"]
+        setattr(p, name, (ctypes.c_int64 * 3)(L * H * base["d"], H * base["d"], base["d"]))
+    return p
+
+
+@pytest.mark.parametrize("bad", [dict(T=65), dict(S=0), dict(d=96), dict(Hq=3), dict(Hkv=128, Hq=128), dict(B=-1),
+                                 dict(sm_scale=0.0), dict(q_pos0=-1)])
+def test_invalid_params_rejected_on_the_host(bad):
+    p = _params(**bad)
+    m = np.zeros(128, dtype=np.uint8)
+    L = sa.lib()
+    dummy = ctypes.c_void_p(4096)
+    assert L.seg_attn_fwd(ctypes.byref(p), dummy, dummy, dummy, m.ctypes.data, dummy, dummy, None, 0, None) == 1
+    assert L.seg_attn_workspace_bytes(ctypes.byref(p), 1) == 0
+    assert L.seg_attn_count_pairs(ctypes.byref(p), m.ctypes.data, None, None, None) == 1
+
+
+def test_null_and_misaligned_pointers_rejected():
+    p = _params()
+    m = np.zeros(2, dtype=np.uint8)
+    L = sa.lib()
+    ok = ctypes.c_void_p(4096)
+    assert L.seg_attn_fwd(ctypes.byref(p), None, ok, ok, m.ctypes.data, ok, ok, None, 0, None) == 1
+    assert L.seg_attn_fwd(ctypes.byref(p), ctypes.c_void_p(4100), ok, ok, m.ctypes.data, ok, ok, None, 0, None) == 1
+    assert L.seg_attn_fwd(ctypes.byref(p), ok, ok, ok, None, ok, ok, None, 0, None) == 1
+    p2 = _params()
+    p2.k_stride = (ctypes.c_int64 * 3)(256 * 2 * 128, 2 * 128 + 4, 128)      # not a multiple of 8 elements
+    assert L.seg_attn_fwd(ctypes.byref(p2), ok, ok, ok, m.ctypes.data, ok, ok, None, 0, None) == 1
+    # backward without (enough) workspace
+    assert L.seg_attn_bwd(ctypes.byref(p), ok, ok, ok, ok, ok, ok, m.ctypes.data, ok, ok, ok, None, 0, None) == 5
+    assert L.seg_attn_bwd(ctypes.byref(p), ok, ok, ok, ok, ok, ok, m.ctypes.data, ok, ok, ok, ok, 16, None) == 5
+
+
+def test_workspace_sizes():
+    p = _params(B=2, Lq=1000, Hq=4)
+    assert sa.workspace_bytes(p, False) == 0
+    assert sa.workspace_bytes(p, True) == (2 * 4 * 1000 * 4 + 255) // 256 * 256
+    assert sa.lib().seg_attn_host_arena_bytes(ctypes.byref(p)) > 0
+
+
+def test_no_device_means_an_error_not_a_fallback():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    p = _params()
+    m = np.zeros(2, dtype=np.uint8)
+    ok = ctypes.c_void_p(4096)
+    st = sa.lib().seg_attn_fwd(ctypes.byref(p), ok, ok, ok, m.ctypes.data, ok, ok, None, 0, None)
+    assert st in (2, 3)      # unsupported device / CUDA error: never a silent CPU path
+
+
+@pytest.mark.parametrize("B,L,Hq,Hkv,S,T,mask", [
+    (1, 2048, 4, 4, 512, 128, [0, 0, 0, 0]),
+    (2, 1000, 4, 2, 200, 72, [1, 0]),
+    (1, 777, 2, 2, 64, 64, [0, 1]),
+    (1, 300, 2, 1, 7, 0, [0]),
+])
+def test_pair_counter_matches_oracle_enumeration(B, L, Hq, Hkv, S, T, mask):
+    nv, nd, tiles = sa.count_pairs(B, L, Hq, Hkv, 128, S, T, mask)
+    assert (nv, nd) == oracle.count_pairs(B, L, Hq, Hkv, S, T, mask)
+    assert tiles * 128 * 128 >= nv
+
+
+def test_benchmark_configuration_counts():
+    for w, want in ((workloads.CONFIGS[0], 2887680), (workloads.CONFIGS[1], 3305635840),
+                    (workloads.CONFIGS[2], 10133962752), (workloads.CONFIGS[3], 87646273536)):
+        m = workloads.head_past_mask(w.Hkv, w.past_frac, w.seed)
+        assert sa.count_pairs(w.B, w.L, w.Hq, w.Hkv, w.d, w.S, w.T, m)[0] == want
+
+
+def test_prefill_state_size_and_validation():
+    pf_params = _params(B=1, Lq=128, kv_len=1024, S=128, T=64, Hq=4, Hkv=2)
+    m = np.array([1, 0], dtype=np.uint8)
+    L = sa.lib()
+    n = L.seg_prefill_state_bytes(ctypes.byref(pf_params), m.ctypes.data)
+    assert n == 2 * (1 * 1 * 1024 * 128 * 2) + 2 * (1 * 1 * (128 + 64) * 128 * 2)
+    bad = _params(B=1, Lq=64, kv_len=1024, S=128, T=64)
+    assert L.seg_prefill_state_bytes(ctypes.byref(bad), m.ctypes.data) == 0
+    h = ctypes.c_void_p()
+    assert L.seg_prefill_create(ctypes.byref(pf_params), m.ctypes.data, None, 0, ctypes.byref(h)) == 5

@@ -1,0 +1,202 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs - element by element on small and mid-size cases, on oracle-computable
+sub-problems at the full benchmark sizes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+import paper_2605_11744_b200 as sa
+from util import (TOL_GRAD, assert_fwd_close, assert_grads_close, f64, group_slices, oracle_rows, oracle_window,
+                  rand_inputs, rel_l2)
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [
+    # B, L, Hq, Hkv, d, S, T, mask
+    (1, 128, 1, 1, 128, 128, 0, [0]),                 # one tile
+    (1, 384, 2, 1, 128, 128, 128, [0]),               # tail = whole previous segment
+    (1, 1024, 4, 2, 128, 256, 128, [0, 1]),           # GQA, mixed flags
+    (2, 700, 4, 2, 128, 200, 72, [1, 0]),             # nothing aligned to the 128 tile, ragged end
+    (1, 1000, 2, 2, 128, 1000, 0, [0, 0]),            # S >= L: plain causal
+    (1, 640, 2, 1, 128, 128, 0, [0]),                 # T = 0: block diagonal
+    (1, 640, 2, 2, 128, 64, 64, [1, 1]),              # segments shorter than a tile, all flagged
+    (1, 333, 2, 2, 64, 100, 100, [0, 1]),             # d = 64, ragged
+    (1, 130, 1, 1, 64, 7, 3, [0]),                    # tiny segments
+    (3, 1, 2, 1, 128, 4, 2, [1]),                     # a single query row
+]
+
+
+@pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask", SMALL)
+def test_small_cases_match_oracle_elementwise(B, L, Hq, Hkv, d, S, T, mask):
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=L + S)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, mask)
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask)
+    assert_fwd_close(O, LSE, Oo, LSEo, "fwd")
+    assert_grads_close((dQ, dK, dV), ref, "bwd")
+
+
+def test_configuration_1_in_full():
+    w = workloads.CONFIGS[0]
+    x = workloads.make_inputs(w)
+    Q, K, V, dO = (x[k].cuda() for k in ("Q", "K", "V", "dO"))
+    O, LSE = sa.seg_attn_fwd(Q, K, V, w.S, w.T, x["mask"], w.sm_scale)
+    grads = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, w.S, w.T, x["mask"], w.sm_scale)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), w.S, w.T, x["mask"])
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), w.S, w.T, x["mask"])
+    assert_fwd_close(O, LSE, Oo, LSEo, w.name)
+    assert_grads_close(grads, ref, w.name)
+
+
+def test_structural_zeros_and_reproducibility():
+    # loss on the third segment only: dK/dV are exactly zero before the tail of segment 2 and after segment 3
+    B, L, Hq, Hkv, d, S, T = 1, 1024, 4, 2, 128, 256, 128
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=5)
+    dO[:, :2 * S] = 0
+    dO[:, 3 * S:] = 0
+    mask = [1, 0]
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask)
+    for G in (dK, dV):
+        assert torch.count_nonzero(G[:, :2 * S - T]) == 0
+        assert torch.count_nonzero(G[:, 3 * S:]) == 0
+        assert torch.count_nonzero(G[:, 2 * S - T:3 * S]) > 0
+    assert torch.count_nonzero(dQ[:, :2 * S]) == 0 and torch.count_nonzero(dQ[:, 3 * S:]) == 0
+    # no atomics anywhere: a second run gives the same bits
+    O2, LSE2 = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    dQ2, dK2, dV2 = sa.seg_attn_bwd(Q, K, V, O2, LSE2, dO, S, T, mask)
+    for a, b in ((O, O2), (LSE, LSE2), (dQ, dQ2), (dK, dK2), (dV, dV2)):
+        assert torch.equal(a, b)
+
+
+def test_unflagged_heads_ignore_everything_before_the_tail():
+    B, L, Hq, Hkv, d, S, T = 1, 1024, 2, 2, 128, 256, 128
+    Q, K, V, _ = rand_inputs(B, L, Hq, Hkv, d, seed=9)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, [0, 1])
+    K2, V2 = K.clone(), V.clone()
+    K2[:, :2 * S - T, 0] = float("nan")  # never staged for the unflagged head's later segments
+    V2[:, :2 * S - T, 0] = float("nan")
+    K2[:, :2 * S - T, 1] += 3.0
+    V2[:, :2 * S - T, 1] -= 2.0
+    O2, LSE2 = sa.seg_attn_fwd(Q, K2, V2, S, T, [0, 1])
+    assert torch.equal(O[:, 2 * S:, 0], O2[:, 2 * S:, 0]) and torch.equal(LSE[:, 0, 2 * S:], LSE2[:, 0, 2 * S:])
+    assert (O[:, 2 * S:, 1].float() - O2[:, 2 * S:, 1].float()).abs().max() > 1e-2   # the flagged head does read them
+
+
+def test_outputs_outside_the_problem_are_untouched_and_strides_respected():
+    # O, dQ, dK, dV live inside larger poisoned buffers (head and position padding)
+    B, L, Hq, Hkv, d, S, T = 2, 300, 2, 1, 128, 128, 64
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=11)
+
+    def padded(t):
+        big = torch.full((t.shape[0], t.shape[1] + 3, t.shape[2] + 1, t.shape[3]), float("nan"),
+                         dtype=t.dtype, device=t.device)
+        view = big[:, :t.shape[1], :t.shape[2]]
+        view.copy_(t)
+        return big, view
+
+    _, Qv = padded(Q)
+    _, Kv = padded(K)
+    _, Vv = padded(V)
+    Obig, Ov = padded(torch.zeros_like(Q))
+    Obig.fill_(float("nan"))
+    O, LSE = sa.seg_attn_fwd(Qv, Kv, Vv, S, T, [1], out=Ov)
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, [1])
+    assert_fwd_close(Ov, LSE, Oo, LSEo, "strided")
+    assert torch.isnan(Obig[:, L:]).all() and torch.isnan(Obig[:, :, Hq:]).all()
+
+
+def test_empty_and_degenerate_shapes():
+    mk = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device="cuda")
+    # no batch, no rows: nothing to do, no error
+    for B, L in ((0, 128), (2, 0)):
+        O, LSE = sa.seg_attn_fwd(mk(B, L, 2, 128), mk(B, L, 1, 128), mk(B, L, 1, 128), 64, 16, [0])
+        dQ, dK, dV = sa.seg_attn_bwd(mk(B, L, 2, 128), mk(B, L, 1, 128), mk(B, L, 1, 128), O, LSE,
+                                     mk(B, L, 2, 128), 64, 16, [0])
+        assert O.numel() == 0 and dK.numel() == 0
+    # keys that do not reach the queries: rows without any visible key give O = 0, LSE = -inf, zero gradients
+    Q, K, V, dO = rand_inputs(1, 256, 2, 1, 128, seed=3, Lk=100)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, 64, 16, [0])
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, 64, 16, [0])
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), 64, 16, [0])
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), 64, 16, [0])
+    assert_fwd_close(O, LSE, Oo, LSEo, "short kv")
+    assert torch.isinf(LSE[:, :, 128:]).all() and torch.count_nonzero(O[:, 128:]) == 0
+    assert_grads_close((dQ, dK, dV), ref, "short kv")
+    assert torch.count_nonzero(dQ[:, 128:]) == 0
+
+
+def test_invalid_arguments_are_rejected_before_launch():
+    Q, K, V, dO = rand_inputs(1, 128, 2, 1, 128)
+    with pytest.raises(sa.SegAttnError) as e:
+        sa.seg_attn_fwd(Q, K, V, 64, 65, [0])                      # T > S
+    assert e.value.status == 1
+    with pytest.raises(sa.SegAttnError):
+        sa.seg_attn_fwd(Q[..., :96].contiguous(), K[..., :96].contiguous(), V[..., :96].contiguous(), 64, 0, [0])
+    O, LSE = sa.seg_attn_fwd(Q, K, V, 64, 16, [0])
+    with pytest.raises(sa.SegAttnError) as e:
+        sa.seg_attn_bwd(Q, K, V, O, LSE, dO, 64, 16, [0], workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 5                                      # workspace too small
+
+
+def _full_size_check(w, late_rows=24, seg_lo=1):
+    x = workloads.make_inputs(w, device="cuda")
+    O, LSE = sa.seg_attn_fwd(x["Q"], x["K"], x["V"], w.S, w.T, x["mask"], w.sm_scale)
+    grads = None
+    if w.backward:
+        grads = sa.seg_attn_bwd(x["Q"], x["K"], x["V"], O, LSE, x["dO"], w.S, w.T, x["mask"], w.sm_scale)
+    sa.poll_status()
+    g = w.Hq // w.Hkv
+    b = w.B - 1
+    rng = np.random.default_rng(w.seed + 1)
+    for c, hq in group_slices(x["mask"], g):
+        ref = oracle_window(x, w, b, c, hq, seg_lo)
+        rows = ref["rows"]
+        assert_fwd_close(O[b:b + 1, rows, hq], LSE[b:b + 1, hq, rows], ref["O"], ref["LSE"], "%s window kv%d" % (w.name, c))
+        if grads is not None:
+            dQ, dK, dV = grads
+            keys = ref["keys"]
+            assert_grads_close((dQ[b:b + 1, rows, hq], dK[b:b + 1, keys, c:c + 1], dV[b:b + 1, keys, c:c + 1]),
+                               (ref["dQ"], ref["dK"], ref["dV"]), "%s window kv%d" % (w.name, c))
+        # rows sampled from the last segment, where a flagged head's visible range is longest
+        last0 = (w.L - 1) // w.S * w.S
+        ps = sorted(set(int(p) for p in rng.integers(last0, w.L, size=late_rows)) | {w.L - 1, last0})
+        num = den = 0.0
+        for p, Oo, LSEo, dQo in oracle_rows(x, w, b, c, hq, ps):
+            assert_fwd_close(O[b:b + 1, p:p + 1, hq], LSE[b:b + 1, hq, p:p + 1], Oo, LSEo, "%s row %d" % (w.name, p))
+            if dQo is not None:
+                num += float(((f64(grads[0][b:b + 1, p:p + 1, hq]) - dQo) ** 2).sum())
+                den += float((dQo ** 2).sum())
+        if grads is not None:
+            assert (num / den) ** 0.5 <= TOL_GRAD, "%s late rows dQ" % w.name
+
+
+def test_configuration_2_full_size_sampled():
+    _full_size_check(workloads.CONFIGS[1])
+
+
+def test_configuration_3_full_size_sampled_with_outlier_keys():
+    _full_size_check(workloads.CONFIGS[2], late_rows=12)
+
+
+@pytest.mark.parametrize("S,T,frac", [(1024, 256, 0.25), (4096, 4096, 0.0), (16384, 1024, 1.0)])
+def test_configuration_5_sweep_points_sampled(S, T, frac):
+    w = workloads.CONFIGS[4].with_(S=S, T=T, past_frac=frac, name="cfg5_S%d_T%d_f%g" % (S, T, frac))
+    _full_size_check(w, late_rows=6, seg_lo=1 if S <= 4096 else 0)
+
+
+def test_host_buffer_step_matches_device_path():
+    w = workloads.CONFIGS[0]
+    x = workloads.make_inputs(w)
+    outs = sa.seg_attn_step_host(x["Q"], x["K"], x["V"], x["dO"], w.S, w.T, x["mask"], w.sm_scale)
+    Q, K, V, dO = (x[k].cuda() for k in ("Q", "K", "V", "dO"))
+    O, LSE = sa.seg_attn_fwd(Q, K, V, w.S, w.T, x["mask"], w.sm_scale)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, w.S, w.T, x["mask"], w.sm_scale)
+    for k, t in (("O", O), ("LSE", LSE), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+        assert torch.equal(outs[k], t.cpu()), k

@@ -1,0 +1,83 @@
+"""Streamed prefill on the GPU: equals the one-shot forward (the forward identity between
+segment-by-segment and whole-sequence execution) and the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+import paper_2605_11744_b200 as sa
+from util import assert_fwd_close, f64, group_slices, oracle_rows, rand_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def run_streamed(Q, K, V, S, T, mask, scale=None):
+    B, L, Hq, d = Q.shape
+    Hkv = K.shape[2]
+    pf = sa.Prefill(B, S, T, Hq, Hkv, d, L, mask, scale)
+    O = torch.empty_like(Q)
+    LSE = torch.empty(B, Hq, L, dtype=torch.float32, device=Q.device)
+    for i in range(L // S):
+        sl = slice(i * S, (i + 1) * S)
+        o, l = pf.step(Q[:, sl].contiguous(), K[:, sl].contiguous(), V[:, sl].contiguous())
+        O[:, sl] = o
+        LSE[:, :, sl] = l
+    sa.poll_status()
+    state = pf.state_bytes
+    pf.close()
+    return O, LSE, state
+
+
+@pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask", [
+    (1, 1024, 4, 2, 128, 256, 128, [0, 1]),
+    (2, 768, 4, 4, 128, 256, 0, [1, 0, 0, 1]),
+    (1, 800, 2, 2, 64, 200, 72, [0, 1]),        # tiles of the window do not line up with the one-shot tiles
+    (1, 512, 2, 2, 128, 128, 128, [0, 0]),
+    (1, 512, 2, 1, 128, 128, 64, [1]),
+])
+def test_streamed_equals_one_shot_and_oracle(B, L, Hq, Hkv, d, S, T, mask):
+    Q, K, V, _ = rand_inputs(B, L, Hq, Hkv, d, seed=L + T)
+    O1, LSE1 = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    O2, LSE2, _ = run_streamed(Q, K, V, S, T, mask)
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, mask)
+    assert_fwd_close(O2, LSE2, Oo, LSEo, "streamed")
+    if S % 128 == 0 and T % 128 == 0:
+        # same tiles in the same order: the two paths agree to the bit
+        assert torch.equal(O1, O2) and torch.equal(LSE1, LSE2)
+    else:
+        assert (O1.float() - O2.float()).abs().max() <= 2e-2
+
+
+def test_reset_and_reuse():
+    Q, K, V, _ = rand_inputs(1, 512, 2, 2, 128, seed=1)
+    pf = sa.Prefill(1, 128, 128, 2, 2, 128, 512, [0, 1])
+    outs = []
+    for rep in range(2):
+        o = [pf.step(Q[:, i * 128:(i + 1) * 128].contiguous(), K[:, i * 128:(i + 1) * 128].contiguous(),
+                     V[:, i * 128:(i + 1) * 128].contiguous())[0] for i in range(4)]
+        outs.append(torch.cat(o, dim=1))
+        with pytest.raises(sa.SegAttnError):
+            pf.step(Q[:, :128].contiguous(), K[:, :128].contiguous(), V[:, :128].contiguous())   # pool is full
+        pf.reset()
+    assert torch.equal(outs[0], outs[1])
+    pf.close()
+
+
+def test_configuration_4_streamed_at_full_size_sampled():
+    w = workloads.CONFIGS[3]
+    x = workloads.make_inputs(w, device="cuda")
+    torch.cuda.synchronize()
+    O, LSE, state = run_streamed(x["Q"], x["K"], x["V"], w.S, w.T, x["mask"], w.sm_scale)
+    # persistent state: the flagged heads' whole history plus the other heads' tail + segment window
+    nf = int(x["mask"].sum())
+    expect = 2 * w.B * nf * w.L * w.d * 2 + 2 * w.B * (w.Hkv - nf) * (w.S + w.T) * w.d * 2
+    assert state == expect
+    O1, LSE1 = sa.seg_attn_fwd(x["Q"], x["K"], x["V"], w.S, w.T, x["mask"], w.sm_scale)
+    assert torch.equal(O, O1) and torch.equal(LSE, LSE1)
+    g = w.Hq // w.Hkv
+    rng = np.random.default_rng(4)
+    for c, hq in group_slices(x["mask"], g):
+        ps = sorted(set(int(p) for p in rng.integers(0, w.L, size=10)) | {0, w.S - 1, w.S, w.L - 1})
+        for p, Oo, LSEo, _ in oracle_rows(x, w, 0, c, hq, ps):
+            assert_fwd_close(O[:, p:p + 1, hq], LSE[:, hq, p:p + 1], Oo, LSEo, "cfg4 row %d kv%d" % (p, c))
