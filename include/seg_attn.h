@@ -151,6 +151,15 @@ int seg_attn_last_cuda_error(void);
  * forward kernel visits.  Any of the output pointers may be NULL. */
 segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* head_past_mask,
                                     int64_t* pairs_visible, int64_t* pairs_diff, int64_t* fwd_tiles);
+/* Measurement aid (the paper has no counterpart): runs each of the four kernels of a training
+ * step on its own - forward, row dots, dQ pass, dK/dV pass, in that order - once untimed and then
+ * `iters` times back to back between two CUDA events recorded on `stream`, and returns the average
+ * milliseconds per launch in ms_per_launch[0..3].  Arguments as for seg_attn_fwd / seg_attn_bwd
+ * (O and LSE are written by the forward and read by the backward).  Synchronises `stream`. */
+segattn_status seg_attn_profile_kernels(const seg_attn_params* p, const void* Q, const void* K, const void* V,
+                                       void* O, float* LSE, const void* dO, const uint8_t* head_past_mask, void* dQ,
+                                       void* dK, void* dV, void* workspace, size_t workspace_bytes, int iters,
+                                       float ms_per_launch[4], void* stream);
 /* Number of kernel launches the library has enqueued so far in this process. */
 int64_t seg_attn_launch_count(void);
 

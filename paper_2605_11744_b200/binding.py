@@ -58,6 +58,8 @@ def lib():
         L.seg_attn_host_arena_bytes.restype = ctypes.c_size_t
         L.seg_attn_host_arena_bytes.argtypes = [pp]
         L.seg_attn_step_host.argtypes = [pp, vp, vp, vp, vp, u8p, vp, fp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.seg_attn_profile_kernels.argtypes = [pp, vp, vp, vp, vp, fp, vp, u8p, vp, vp, vp, vp, ctypes.c_size_t,
+                                               ctypes.c_int, ctypes.POINTER(ctypes.c_float * 4), vp]
         L.seg_attn_poll_status.argtypes = [vp]
         L.seg_attn_status_string.restype = ctypes.c_char_p
         L.seg_attn_status_string.argtypes = [ctypes.c_int]
@@ -175,6 +177,24 @@ def seg_attn_step_host(Q, K, V, dO, S: int, T: int, head_past_mask=None, sm_scal
                                     ctypes.c_void_p(arena.data_ptr()), arena.numel(), _stream(stream)),
            "seg_attn_step_host")
     return outs
+
+
+def profile_kernels(Q, K, V, dO, S: int, T: int, head_past_mask=None, sm_scale=None, iters: int = 5, stream=None):
+    """Average milliseconds per launch of (forward, row dots, dQ pass, dK/dV pass), each timed on its own
+    with CUDA events on the launching stream by the C entry point `seg_attn_profile_kernels`."""
+    _need_cuda_bf16(Q, K, V, dO)
+    O = torch.empty_like(Q)
+    LSE = torch.empty((Q.shape[0], Q.shape[2], Q.shape[1]), dtype=torch.float32, device=Q.device)
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    p = params_for(Q, K, V, O, S, T, sm_scale)
+    m = _mask_arr(head_past_mask, p.Hkv)
+    ws = torch.empty(max(workspace_bytes(p, True), 256), dtype=torch.uint8, device=Q.device)
+    ms = (ctypes.c_float * 4)()
+    _check(lib().seg_attn_profile_kernels(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), _ptr(dO),
+                                          m.ctypes.data, _ptr(dQ), _ptr(dK), _ptr(dV), ctypes.c_void_p(ws.data_ptr()),
+                                          ws.numel(), iters, ctypes.byref(ms), _stream(stream)),
+           "seg_attn_profile_kernels")
+    return {"fwd": ms[0], "rowdot": ms[1], "dq": ms[2], "dkv": ms[3]}
 
 
 class Prefill:
