@@ -7,6 +7,8 @@
 // owner, warps 2..5 element-wise work with one thread per accumulator row.  No atomics: a CTA
 // owns its output tile, so results are bitwise reproducible.
 #pragma once
+#include <type_traits>
+
 #include "mask.cuh"
 #include "ptx.cuh"
 
@@ -215,6 +217,47 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
             dsum = prm.Dvec[sidx];
         }
         const float sl2 = prm.scale_log2;
+        const uint64_t sl2x2 = f32x2(sl2, sl2);
+        const uint64_t nlse2 = f32x2(-lse2, -lse2);
+        const uint64_t ndsum2 = f32x2(-dsum, -dsum);
+        // dS = P * (dP - D) for one key tile; MASKED is a compile-time flag so that fully visible
+        // tiles run branch-free straight-line code
+        auto ds_tile = [&](auto masked_c, const int c0) {
+            constexpr bool MASKED = decltype(masked_c)::value;
+            uint32_t sa_[32], sb_[32], da_[32], db_[32];
+            tmem_ld_x32(tS + lane_off, sa_);
+            tmem_ld_x32(tDp + lane_off, da_);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t(&sv)[32] = (c & 1) ? sb_ : sa_;
+                uint32_t(&dv)[32] = (c & 1) ? db_ : da_;
+                uint32_t(&sn)[32] = (c & 1) ? sa_ : sb_;
+                uint32_t(&dn)[32] = (c & 1) ? da_ : db_;
+                tmem_wait_ld_dep(sv);
+                tmem_wait_ld_dep(dv);
+                if (c < 3) {
+                    tmem_ld_x32(tS + lane_off + (c + 1) * 32, sn);
+                    tmem_ld_x32(tDp + lane_off + (c + 1) * 32, dn);
+                }
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float t0, t1;
+                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[i], sv[i + 1]), sl2x2, nlse2), t0, t1);
+                    const uint64_t p2 = f32x2(ex2(t0), ex2(t1));
+                    const uint64_t ds2 = mul_f32x2(p2, add_f32x2(f32x2_bits(dv[i], dv[i + 1]), ndsum2));
+                    float d0, d1;
+                    f32x2_unpack(ds2, d0, d1);
+                    if (MASKED) {
+                        const int col = c0 + c * 32 + i;
+                        d0 = (col >= vlo && col <= vhi) ? d0 : 0.f;
+                        d1 = (col + 1 >= vlo && col + 1 <= vhi) ? d1 : 0.f;
+                    }
+                    pk[i / 2] = pack_bf16(d0, d1);
+                }
+                tmem_st_x16(tDs + lane_off + c * 16, pk);
+            }
+        };
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int c0 = (t_lo + j) * kTile;
@@ -222,28 +265,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
             ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), j & 1, 17));
             if (!ok) break;
             tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t sv[32], dv[32];
-                tmem_ld_x32(tS + lane_off + c * 32, sv);
-                tmem_ld_x32(tDp + lane_off + c * 32, dv);
-                tmem_wait_ld();
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float p0 = ex2(fmaf(__uint_as_float(sv[i]), sl2, -lse2));
-                    float p1 = ex2(fmaf(__uint_as_float(sv[i + 1]), sl2, -lse2));
-                    float d0 = p0 * (__uint_as_float(dv[i]) - dsum);
-                    float d1 = p1 * (__uint_as_float(dv[i + 1]) - dsum);
-                    if (masked) {
-                        const int col = c0 + c * 32 + i;
-                        if (!(col >= vlo && col <= vhi)) d0 = 0.f;
-                        if (!(col + 1 >= vlo && col + 1 <= vhi)) d1 = 0.f;
-                    }
-                    pk[i / 2] = pack_bf16(d0, d1);
-                }
-                tmem_st_x16(tDs + lane_off + c * 16, pk);
-            }
+            if (masked) ds_tile(std::true_type{}, c0);
+            else ds_tile(std::false_type{}, c0);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(kBarDsFull));
@@ -445,6 +468,49 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
                 d_next = prm.Dvec[si];
             }
         }
+        const uint64_t sl2x2 = f32x2(sl2, sl2);
+        // P^T = 2^(S^T*scale*log2e - LSE_q*log2e) and dS^T = P^T * (dP^T - D_q) for one query tile
+        // (query = column); MASKED is a compile-time flag so that full tiles run branch-free code
+        auto pt_tile = [&](auto masked_c, const int buf, const int q0) {
+            constexpr bool MASKED = decltype(masked_c)::value;
+            uint32_t sa_[32], sb_[32], da_[32], db_[32];
+            tmem_ld_x32(tSt + lane_off, sa_);
+            tmem_ld_x32(tDpt + lane_off, da_);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t(&sv)[32] = (c & 1) ? sb_ : sa_;
+                uint32_t(&dv)[32] = (c & 1) ? db_ : da_;
+                uint32_t(&sn)[32] = (c & 1) ? sa_ : sb_;
+                uint32_t(&dn)[32] = (c & 1) ? da_ : db_;
+                tmem_wait_ld_dep(sv);
+                tmem_wait_ld_dep(dv);
+                if (c < 3) {
+                    tmem_ld_x32(tSt + lane_off + (c + 1) * 32, sn);
+                    tmem_ld_x32(tDpt + lane_off + (c + 1) * 32, dn);
+                }
+                uint32_t pk[16], dk[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    const float2 l2 = *reinterpret_cast<const float2*>(&s_lse[buf][c * 32 + e]);
+                    const float2 dd = *reinterpret_cast<const float2*>(&s_dsum[buf][c * 32 + e]);
+                    float t0, t1;
+                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[e], sv[e + 1]), sl2x2, f32x2(-l2.x, -l2.y)), t0, t1);
+                    float p0 = ex2(t0), p1 = ex2(t1);
+                    if (MASKED) {
+                        const int q = q0 + c * 32 + e;
+                        p0 = (q >= qlo && q <= qhi) ? p0 : 0.f;
+                        p1 = (q + 1 >= qlo && q + 1 <= qhi) ? p1 : 0.f;
+                    }
+                    const uint64_t ds2 = mul_f32x2(f32x2(p0, p1), add_f32x2(f32x2_bits(dv[e], dv[e + 1]), f32x2(-dd.x, -dd.y)));
+                    float d0, d1;
+                    f32x2_unpack(ds2, d0, d1);
+                    pk[e / 2] = pack_bf16(p0, p1);
+                    dk[e / 2] = pack_bf16(d0, d1);
+                }
+                tmem_st_x16(tPt + lane_off + c * 16, pk);
+                tmem_st_x16(tDst + lane_off + c * 16, dk);
+            }
+        };
         bool ok = true;
         for (int i = 0; i < n_it; ++i) {
             const int buf = i & 1;
@@ -468,32 +534,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), i & 1, 25));
             if (!ok) continue;
             tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t sv[32], dv[32];
-                tmem_ld_x32(tSt + lane_off + c * 32, sv);
-                tmem_ld_x32(tDpt + lane_off + c * 32, dv);
-                tmem_wait_ld();
-                uint32_t pk[16], dk[16];
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    const float2 l2 = *reinterpret_cast<const float2*>(&s_lse[buf][c * 32 + e]);
-                    const float2 dd = *reinterpret_cast<const float2*>(&s_dsum[buf][c * 32 + e]);
-                    float p0 = ex2(fmaf(__uint_as_float(sv[e]), sl2, -l2.x));
-                    float p1 = ex2(fmaf(__uint_as_float(sv[e + 1]), sl2, -l2.y));
-                    if (masked) {
-                        const int q = q0 + c * 32 + e;
-                        if (!(q >= qlo && q <= qhi)) p0 = 0.f;
-                        if (!(q + 1 >= qlo && q + 1 <= qhi)) p1 = 0.f;
-                    }
-                    const float d0 = p0 * (__uint_as_float(dv[e]) - dd.x);
-                    const float d1 = p1 * (__uint_as_float(dv[e + 1]) - dd.y);
-                    pk[e / 2] = pack_bf16(p0, p1);
-                    dk[e / 2] = pack_bf16(d0, d1);
-                }
-                tmem_st_x16(tPt + lane_off + c * 16, pk);
-                tmem_st_x16(tDst + lane_off + c * 16, dk);
-            }
+            if (masked) pt_tile(std::true_type{}, buf, q0);
+            else pt_tile(std::false_type{}, buf, q0);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(kBarPFull));

@@ -7,6 +7,8 @@
 // TMEM (256 columns): S / P at columns [0,128) (P, bf16, aliases the first 64), O at [128,128+D).
 // Two CTAs are resident per SM so that one CTA's softmax overlaps the other's MMAs.
 #pragma once
+#include <type_traits>
+
 #include "mask.cuh"
 #include "ptx.cuh"
 
@@ -150,15 +152,19 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
                 ok = mbar_wait(bar(kBarPFull), j & 1, 5) && mbar_wait(bar(kBarVFull), j & 1, 6);
                 if (!ok) break;
                 tc_fence_after();
+                TRACE(true, j * 8 + 4);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
                     mma_ts(tO, tP + k * 8, make_sdesc(sV + k * 2048, 16384, 1024), idesc_pv, (j > 0) || (k > 0));
                 mma_commit(bar(kBarVEmpty));
+                TRACE(true, j * 8 + 5);
                 if (j + 1 < n_tiles) {
                     ok = mbar_wait(bar(kBarKFull), (j + 1) & 1, 7);
                     if (!ok) break;
                     tc_fence_after();
+                    TRACE(true, j * 8 + 6);
                     issue_qk();
+                    TRACE(true, j * 8 + 7);
                     mma_commit(bar(kBarKEmpty));
                     mma_commit(bar(kBarSFull));
                 } else {
@@ -184,36 +190,43 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
         if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
 
         const float sl2 = prm.scale_log2;
-        // l_run: row sum of the unrounded p (gives LSE); lr_run: row sum of the bf16-rounded p that
-        // the PV product actually uses, so that O = sum(p~ v) / sum(p~) stays a convex combination
-        // of value rows even when one key dominates (outlier keys)
-        float m_run = -INFINITY, l_run = 0.f, lr_run = 0.f;
+        const uint64_t sl2x2 = f32x2(sl2, sl2);
+        // l_run: row sum of the unrounded p (gives LSE).  c_run: sum over tiles of (bf16(p) - p) for the
+        // tile's largest p.  O is divided by l_run + c_run, i.e. by a row sum in which the dominant
+        // probability enters as the bf16 value the PV product really used, so that a row where one key
+        // dominates (outlier keys) stays a convex combination of value rows.
+        float m_run = -INFINITY, l_run = 0.f, c_run = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int c0 = (t_lo + j) * kTile;
-            const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), j & 1, 8));
-            if (!ok) break;
-            tc_fence_after();
-            // pass 1: row maximum of the raw scores
-            float mx = -INFINITY;
+        // One key tile of the online softmax.  MASKED is a compile-time flag so that the common,
+        // fully visible tile runs straight-line code (no per-element tests, no branches that would keep
+        // the scheduler from overlapping the exp latency of neighbouring elements).
+        auto softmax_tile = [&](auto masked_c, const int j, const int c0) {
+            constexpr bool MASKED = decltype(masked_c)::value;
+            uint32_t va[32], vb[32];
+            // pass 1: row maximum of the raw scores; the load of chunk c+1 is in flight while chunk c is reduced
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+            tmem_ld_x32(tS + lane_off, va);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld_x32(tS + lane_off + c * 32, v);
-                tmem_wait_ld();
-                if (masked) {
+                uint32_t(&cur)[32] = (c & 1) ? vb : va;
+                uint32_t(&nxt)[32] = (c & 1) ? va : vb;
+                tmem_wait_ld_dep(cur);
+                tmem_ld_x32(tS + lane_off + ((c + 1) & 3) * 32, nxt);  // c == 3: chunk 0 again, for pass 2
+                if (MASKED) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const int col = c0 + c * 32 + i;
-                        const float s = (col >= vlo && col <= vhi) ? __uint_as_float(v[i]) : -INFINITY;
-                        mx = fmaxf(mx, s);
+                        cur[i] = (col >= vlo && col <= vhi) ? cur[i] : 0xff800000u;  // -inf
                     }
-                } else {
+                }
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+                for (int i = 0; i < 32; i += 4) {
+                    mx0 = fmax3(mx0, __uint_as_float(cur[i]), __uint_as_float(cur[i + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(cur[i + 2]), __uint_as_float(cur[i + 3]));
                 }
             }
+            const float mx = fmaxf(mx0, mx1);
+            TRACE(tid == 64, j * 8 + 1);
             const float m_tile = mx * sl2;  // scale > 0, so the maximum commutes with the scaling
             const float m_new = fmaxf(m_run, m_tile);
             const bool grow = m_new > m_run + kRescaleThreshold || (m_run == -INFINITY && m_new > -INFINITY);
@@ -221,16 +234,17 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
             if (grow) {
                 alpha = ex2(m_run - m_new);  // 0 when nothing was accumulated yet
                 l_run *= alpha;
-                lr_run *= alpha;
+                c_run *= alpha;
                 m_run = m_new;
             }
             if (j > 0 && __any_sync(0xffffffffu, grow)) {
                 // every MMA issued before this tile's S (the previous PV included) has retired
+                tmem_wait_ld_dep(va);  // the prefetched chunk 0: drain before reusing the load path
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t v[32];
                     tmem_ld_x32(tO + lane_off + c * 32, v);
-                    tmem_wait_ld();
+                    tmem_wait_ld_dep(v);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
                     tmem_st_x32(tO + lane_off + c * 32, v);
@@ -238,40 +252,62 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
             }
             // pass 2: p = 2^(s*scale*log2e - m); row sum from the unrounded p; P to TMEM as bf16
             const float m_eff = (m_run == -INFINITY) ? 0.f : m_run;
-            float lsum = 0.f, lsum_r = 0.f;
+            const uint64_t nm2 = f32x2(-m_eff, -m_eff);
+            {
+                const float pm = ex2(fmaf(mx, sl2, -m_eff));  // the tile's largest p, exactly as pass 2 forms it
+                const uint32_t pr = pack_bf16(pm, 0.f);
+                c_run += __uint_as_float(pr << 16) - pm;
+            }
+            uint64_t acc_a = 0ull, acc_b = 0ull;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld_x32(tS + lane_off + c * 32, v);
-                tmem_wait_ld();
+                uint32_t(&cur)[32] = (c & 1) ? vb : va;
+                uint32_t(&nxt)[32] = (c & 1) ? va : vb;
+                tmem_wait_ld_dep(cur);
+                if (c < 3) tmem_ld_x32(tS + lane_off + (c + 1) * 32, nxt);
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    float p0 = ex2(fmaf(__uint_as_float(v[i]), sl2, -m_eff));
-                    float p1 = ex2(fmaf(__uint_as_float(v[i + 1]), sl2, -m_eff));
-                    if (masked) {
+                    const uint64_t t = fma_f32x2(f32x2_bits(cur[i], cur[i + 1]), sl2x2, nm2);
+                    float t0, t1;
+                    f32x2_unpack(t, t0, t1);
+                    float p0 = ex2(t0), p1 = ex2(t1);
+                    if (MASKED) {
                         const int col = c0 + c * 32 + i;
-                        if (!(col >= vlo && col <= vhi)) p0 = 0.f;
-                        if (!(col + 1 >= vlo && col + 1 <= vhi)) p1 = 0.f;
+                        p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
+                        p1 = (col + 1 >= vlo && col + 1 <= vhi) ? p1 : 0.f;
                     }
-                    lsum += p0 + p1;
-                    const uint32_t pr = pack_bf16(p0, p1);
-                    lsum_r += __uint_as_float(pr << 16) + __uint_as_float(pr & 0xffff0000u);
-                    pk[i / 2] = pr;
+                    if (i & 2) acc_b = add_f32x2(acc_b, f32x2(p0, p1));
+                    else acc_a = add_f32x2(acc_a, f32x2(p0, p1));
+                    pk[i / 2] = pack_bf16(p0, p1);
                 }
                 tmem_st_x16(tP + lane_off + c * 16, pk);
             }
-            l_run += lsum;
-            lr_run += lsum_r;
+            {
+                float s0, s1;
+                f32x2_unpack(add_f32x2(acc_a, acc_b), s0, s1);
+                l_run += s0 + s1;
+            }
+        };
+        for (int j = 0; j < n_tiles; ++j) {
+            const int c0 = (t_lo + j) * kTile;
+            const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), j & 1, 8));
+            if (!ok) break;
+            tc_fence_after();
+            TRACE(tid == 64, j * 8 + 0);
+            if (masked) softmax_tile(std::true_type{}, j, c0);
+            else softmax_tile(std::false_type{}, j, c0);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(kBarPFull));
+            TRACE(tid == 64, j * 8 + 2);
         }
         // ---------------- epilogue ----------------
         if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), 0, 9));
         tc_fence_after();
-        const bool have = n_tiles > 0 && ok && l_run > 0.f && lr_run > 0.f;
-        const float inv_l = have ? 1.f / lr_run : 0.f;
+        const bool have = n_tiles > 0 && ok && l_run > 0.f && l_run + c_run > 0.f;
+        const float inv_l = have ? 1.f / (l_run + c_run) : 0.f;
         if (r < geo.Lq && (ok || n_tiles == 0)) {
             __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(prm.O) + it.b * prm.o_stride[0] +
                                   (long long)r * prm.o_stride[1] + it.hq * prm.o_stride[2];
@@ -288,7 +324,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_x32(tO + lane_off + c * 32, v);
-                tmem_wait_ld();
+                tmem_wait_ld_dep(v);
                 if (r < geo.Lq && have) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {

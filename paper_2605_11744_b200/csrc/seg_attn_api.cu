@@ -280,3 +280,17 @@ segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* hea
 
 #include "seg_attn_bwd_api.inc"
 #include "seg_attn_prefill_api.inc"
+
+#ifdef SEGATTN_TRACE
+// Debug builds only: choose the traced CTA / read back its clock stamps.
+extern "C" int seg_attn_debug_trace(long long* out, int n, int set_block) {
+    if (set_block >= 0) {
+        static long long zeros[4096];
+        cudaMemcpyToSymbol(g_trace_block, &set_block, sizeof(int));
+        cudaMemcpyToSymbol(g_trace, zeros, sizeof(zeros));
+        return 0;
+    }
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * (n < 4096 ? n : 4096));
+}
+#endif
