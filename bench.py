@@ -223,6 +223,22 @@ def measure_prefill(sa, peaks):
             "tflops": fm["fwd"] / t / 1e12, "frac_of_bf16_peak": fm["fwd"] / t / 1e12 / peaks["bf16"]}
 
 
+def max_over_ranks(value, world, device):
+    """The slowest rank's figure (every multi-GPU number is the maximum over ranks).  The only
+    collective of a multi-GPU run; it is outside the data path."""
+    if world <= 1:
+        return float(value)
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(flops_per_rank_step, world, seconds_per_step):
+    """Whole-job throughput of `world` independent replicas in TFLOP/s."""
+    return world * flops_per_rank_step / seconds_per_step / 1e12
+
+
 def run_ours(args, w):
     import torch.distributed as dist
     import paper_2605_11744_b200 as sa
@@ -276,10 +292,7 @@ def run_ours(args, w):
     ms_total = e0.elapsed_time(e1)
     launches = sa.launch_count() - launches0
     sa.poll_status()
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, "cuda")
 
     # end to end through the host-buffer entry point: pinned host tensors in, pinned host tensors out
     host = {k: x[k].cpu().pin_memory() for k in ("Q", "K", "V") + (("dO",) if w.backward else ())}
@@ -294,10 +307,7 @@ def run_ours(args, w):
                               outs=outs)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, world, "cuda")
     h2d = sum(t.numel() * t.element_size() for t in host.values())
     d2h = sum(t.numel() * t.element_size() for t in outs.values())
     clocks = sampler.stop() if rank == 0 else {}
@@ -331,7 +341,7 @@ def run_ours(args, w):
         if not args.no_prefill:
             prefill = measure_prefill(sa, peaks)
         t_step = ms_total / args.steps / 1e3
-        value = world * flops_step / t_step / 1e12
+        value = aggregate_value(flops_step, world, t_step)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -345,7 +355,7 @@ def run_ours(args, w):
             "frac_of_bf16_peak": value / world / peaks["bf16"],
             "frac_of_bf16_sustained": value / world / peaks["bf16_sustained"],
             "roofline": roofline, "cpu_baseline": cpu,
-            "e2e": {"value": world * flops_step * e2e_steps / e2e_s / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": aggregate_value(flops_step, world, e2e_s / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": launches, "clocks": clocks, "prefill": prefill,
         }

@@ -1,0 +1,48 @@
+"""Host-side logic of a multi-GPU benchmark run, exercised with two gloo ranks on CPU: the
+slowest rank's time is the one reported, the aggregate counts every replica, and the reference
+arm runs on rank 0 only."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def _rank_main(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    ms = bench.max_over_ranks(10.0 + 5.0 * rank, world, "cpu")    # rank 1 is the slow one
+    dist.barrier()
+    if rank == 0:
+        json.dump({"ms": ms, "value": bench.aggregate_value(3e12, world, ms / 1e3)}, open(out, "w"))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_report_the_slowest_time_and_the_whole_job(tmp_path):
+    out = str(tmp_path / "r.json")
+    port = 29500 + os.getpid() % 2000
+    mp.spawn(_rank_main, args=(2, port, out), nprocs=2, join=True)
+    r = json.load(open(out))
+    assert r["ms"] == 15.0
+    assert r["value"] == pytest.approx(2 * 3e12 / 15e-3 / 1e12)
+
+
+def test_single_rank_needs_no_process_group():
+    import bench
+    assert bench.max_over_ranks(7.5, 1, "cpu") == 7.5
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "0", "--config", "1"], env=env, capture_output=True, text=True,
+                       timeout=300)
+    assert r.returncode == 0 and r.stdout.strip() == ""
