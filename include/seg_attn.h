@@ -52,7 +52,8 @@ typedef enum {
     SEGATTN_ERR_UNSUPPORTED_ARCH = 2, /* the current device is not compute capability 10.x */
     SEGATTN_ERR_CUDA = 3,             /* a CUDA runtime/driver call failed; see seg_attn_last_cuda_error() */
     SEGATTN_ERR_TIMEOUT = 4,          /* a bounded wait inside a kernel expired (see seg_attn_poll_status) */
-    SEGATTN_ERR_WORKSPACE = 5         /* workspace/state buffer missing, misaligned or too small */
+    SEGATTN_ERR_WORKSPACE = 5,        /* workspace/state buffer missing, misaligned or too small */
+    SEGATTN_ERR_TOO_LARGE = 6         /* problem exceeds the fixed scratch of seg_attn_bwd_static */
 } segattn_status;
 
 typedef struct {
@@ -102,6 +103,29 @@ segattn_status seg_attn_bwd(const seg_attn_params* p, const void* Q, const void*
                             const void* O, const float* LSE, const void* dO,
                             const uint8_t* head_past_mask, void* dQ, void* dK, void* dV,
                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Backward for callers that cannot allocate device memory (the paper has no counterpart; this is
+ * a packaging variant of seg_attn_bwd, not another operation).  Some hosts of this library may
+ * not call cudaMalloc where the backward runs - a serving or training loop whose memory pool is
+ * sized at start-up and frozen, a plugin that is handed tensors but no allocator, code that must
+ * not trigger the implicit device synchronisation an allocation can cause - and so cannot provide
+ * the `workspace` seg_attn_bwd asks for.  This entry point takes
+ * no workspace: the fp32 row dots D live in a fixed array inside the library's device image,
+ * SEG_ATTN_STATIC_MAX_ROWS floats (4 MiB) that every GPU loading the library holds until the
+ * process exits.  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Same arguments, results and error codes as seg_attn_bwd otherwise (same kernels).
+ *   - Problems with B * Hq * Lq > SEG_ATTN_STATIC_MAX_ROWS are rejected with
+ *     SEGATTN_ERR_TOO_LARGE before anything is launched; use seg_attn_bwd with a workspace.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress, with that device current).  Make that first call outside any stream
+ *     capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents (every
+ *     element a call reads it has written first, so nothing needs clearing).  Two calls whose
+ *     work overlaps on the GPU - different streams, or threads - race on it: serialise them. */
+#define SEG_ATTN_STATIC_MAX_ROWS (1 << 20)
+segattn_status seg_attn_bwd_static(const seg_attn_params* p, const void* Q, const void* K, const void* V,
+                                   const void* O, const float* LSE, const void* dO,
+                                   const uint8_t* head_past_mask, void* dQ, void* dK, void* dV, void* stream);
 
 /* ---- Streamed prefill: the segment recurrence (C_i, o_i) = F(x_i, C_{i-1}, R_{i-1}) of
  * Definition 3.1 restricted to attention, with memory bounded as in Section 3.5 "Memory

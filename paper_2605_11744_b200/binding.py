@@ -48,6 +48,7 @@ def lib():
         L.seg_attn_workspace_bytes.argtypes = [pp, ctypes.c_int]
         L.seg_attn_fwd.argtypes = [pp, vp, vp, vp, u8p, vp, fp, vp, ctypes.c_size_t, vp]
         L.seg_attn_bwd.argtypes = [pp, vp, vp, vp, vp, fp, vp, u8p, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.seg_attn_bwd_static.argtypes = [pp, vp, vp, vp, vp, fp, vp, u8p, vp, vp, vp, vp]
         L.seg_prefill_state_bytes.restype = ctypes.c_size_t
         L.seg_prefill_state_bytes.argtypes = [pp, u8p]
         L.seg_prefill_create.argtypes = [pp, u8p, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
@@ -150,6 +151,31 @@ def seg_attn_bwd(Q, K, V, O, LSE, dO, S: int, T: int, head_past_mask=None, sm_sc
     _check(lib().seg_attn_bwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), _ptr(dO),
                               m.ctypes.data, _ptr(dQ), _ptr(dK), _ptr(dV), ctypes.c_void_p(ws.data_ptr()),
                               ws.numel(), _stream(stream)), "seg_attn_bwd")
+    return dQ, dK, dV
+
+
+STATIC_MAX_ROWS = 1 << 20   # SEG_ATTN_STATIC_MAX_ROWS of the C header
+
+
+def seg_attn_bwd_static(Q, K, V, O, LSE, dO, S: int, T: int, head_past_mask=None, sm_scale=None, q_pos0=0,
+                        kv_pos0=0, out=None, stream=None):
+    """dQ, dK, dV through the C entry point `seg_attn_bwd_static`: the backward for callers that cannot
+    allocate device memory where it runs.  No workspace is passed and none is allocated - the row dots
+    live in a fixed 4 MiB array inside the library, so B*Hq*Lq must not exceed STATIC_MAX_ROWS (larger
+    problems raise SegAttnError, status 6).  Pass `out=(dQ, dK, dV)` to supply the gradient buffers too;
+    otherwise they are the only tensors this wrapper creates.  Calls share the array: do not let two of
+    them overlap on the GPU, and make the first call on a device outside any stream capture."""
+    _need_cuda_bf16(Q, K, V, O, dO)
+    if dO.stride() != O.stride():
+        raise ValueError("dO must have the strides of O")
+    dQ, dK, dV = (torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)) if out is None else out
+    if dQ.stride() != Q.stride() or dK.stride() != K.stride() or dV.stride() != V.stride():
+        raise ValueError("gradients must have the strides of Q, K, V")
+    p = params_for(Q, K, V, O, S, T, sm_scale, q_pos0, kv_pos0)
+    m = _mask_arr(head_past_mask, p.Hkv)
+    _check(lib().seg_attn_bwd_static(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), _ptr(dO),
+                                     m.ctypes.data, _ptr(dQ), _ptr(dK), _ptr(dV), _stream(stream)),
+           "seg_attn_bwd_static")
     return dQ, dK, dV
 
 

@@ -234,6 +234,8 @@ const char* seg_attn_status_string(segattn_status s) {
         case SEGATTN_ERR_CUDA: return "CUDA call failed";
         case SEGATTN_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
         case SEGATTN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SEGATTN_ERR_TOO_LARGE:
+            return "problem exceeds the fixed scratch of seg_attn_bwd_static (B*Hq*Lq > SEG_ATTN_STATIC_MAX_ROWS)";
     }
     return "unknown status";
 }
@@ -280,6 +282,59 @@ segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* hea
 
 #include "seg_attn_bwd_api.inc"
 #include "seg_attn_prefill_api.inc"
+
+// ---- Backward without a caller-provided workspace ---------------------------------------------
+// The row dots D = <dO, O> of seg_attn_bwd_static live here instead of in caller memory.  In host
+// code this name is only a handle for the runtime's symbol calls, never a device address: the
+// address the kernels get comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) float g_static_row_dots[SEG_ATTN_STATIC_MAX_ROWS];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+float* g_static_ptr[kMaxDevices] = {};  // per device: address of g_static_row_dots on that device
+
+// Device address of the static scratch on the current device (first use per device: one symbol look-up).
+segattn_status static_scratch(float** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return SEGATTN_ERR_INVALID;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_row_dots);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (!ptr) return SEGATTN_ERR_CUDA;
+        g_static_ptr[dev] = static_cast<float*>(ptr);
+    }
+    *out = g_static_ptr[dev];
+    return SEGATTN_OK;
+}
+
+}  // namespace
+
+extern "C" segattn_status seg_attn_bwd_static(const seg_attn_params* p, const void* Q, const void* K, const void* V,
+                                              const void* O, const float* LSE, const void* dO,
+                                              const uint8_t* head_past_mask, void* dQ, void* dK, void* dV,
+                                              void* stream) {
+    if (!params_ok(p) || !head_past_mask || !all_strides_ok(p)) return SEGATTN_ERR_INVALID;
+    const bool have_q = p->B > 0 && p->Lq > 0, have_kv = p->B > 0 && p->kv_len > 0;
+    if (have_q && (!Q || !O || !LSE || !dO || !dQ || !aligned16(Q) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
+                   (reinterpret_cast<uintptr_t>(LSE) & 3u)))
+        return SEGATTN_ERR_INVALID;
+    if (have_kv && (!K || !V || !dK || !dV || !aligned16(K) || !aligned16(V) || !aligned16(dK) || !aligned16(dV)))
+        return SEGATTN_ERR_INVALID;
+    if ((long long)p->B * p->Hq * p->Lq > (long long)SEG_ATTN_STATIC_MAX_ROWS) return SEGATTN_ERR_TOO_LARGE;
+    segattn_status st = check_arch();
+    if (st != SEGATTN_OK) return st;
+    float* row_dots = nullptr;
+    if ((st = static_scratch(&row_dots)) != SEGATTN_OK) return st;
+    HeadTable heads;
+    identity_heads(&heads, p->Hkv, head_past_mask);
+    return launch_bwd(p, heads, Q, K, V, O, LSE, dO, dQ, dK, dV, row_dots, static_cast<cudaStream_t>(stream));
+}
 
 #ifdef SEGATTN_TRACE
 // Debug builds only: choose the traced CTA / read back its clock stamps.
