@@ -2,10 +2,13 @@
 //   bwd_rowdot_kernel   D_p = <dO_p, O_p>                                    (HBM-bound)
 //   seg_attn_bwd_dq_kernel    dQ_p = scale * sum_{visible j} dS_pj K_j             (sg keys included)
 //   seg_attn_bwd_dkv_kernel   dK_j = scale * sum_{diff(p,j)} dS_pj Q_p,  dV_j = sum_{diff(p,j)} P_pj dO_p
-// with P = 2^(s*scale*log2e - LSE*log2e), dS = P * (dO V^T - D).  Both tensor-core kernels use
-// the role split of the forward kernel: warp 0 TMA producer, warp 1 tcgen05 issuer and TMEM
-// owner, warps 2..5 element-wise work with one thread per accumulator row.  No atomics: a CTA
-// owns its output tile, so results are bitwise reproducible.
+// with P = 2^(s*scale*log2e - LSE*log2e), dS = P * (dO V^T - D).  Both tensor-core kernels run
+// 384 threads: warp 0 TMA producer, warp 1 tcgen05 issuer and TMEM owner, warps 4..11 element-wise
+// work (warp w owns the 32 accumulator rows of TMEM lane quarter w % 4 and the column half
+// (w - 4) / 4 of every 128-column tile; warps 2, 3 idle).  The element-wise work of a tile is cut in
+// two phases - A: P from the scores, B: dS from P and dP - and the tensor-core issue order is
+// arranged so that each phase runs while the tensor cores work on products that do not depend on
+// it.  No atomics: a CTA owns its output tile, so results are bitwise reproducible.
 #pragma once
 #include <type_traits>
 
@@ -14,7 +17,9 @@
 
 namespace segattn {
 
-constexpr int kBwdThreads = 192;
+constexpr int kBwdThreads = 384;
+constexpr int kEwWarp0 = 4;   // first element-wise warp
+constexpr int kEwWarps = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ------------------------------------------------------------------------------------------
@@ -52,18 +57,38 @@ __global__ void __launch_bounds__(256) bwd_rowdot_kernel(const __nv_bfloat16* __
 }
 
 // ------------------------------------------------------------------------------------------
-// dQ pass.  TMEM (512 columns): S / dS at [0,128) (dS, bf16, aliases the first 64),
-// dP at [128,256), dQ accumulator at [256,256+D).
+// Shared pieces of the two tensor-core kernels.
+
+// One arrival per element-wise warp: every lane has fenced its tensor-memory accesses, the warp
+// converges, one lane arrives.
+__device__ __forceinline__ void ew_warp_arrive(uint32_t bar, int lane) {
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
+__device__ __forceinline__ void ew_bar_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// TMEM column of the bf16 A operand for K-step k (16 elements = 8 packed columns): the two
+// column halves keep their packed values at the start of their own 64-column half, so that a
+// warp never writes over fp32 columns the other half's warp may still have to read.
+__device__ __forceinline__ uint32_t packed_a_col(int k) { return (uint32_t)((k >> 2) * 64 + (k & 3) * 8); }
+
+// ------------------------------------------------------------------------------------------
+// dQ pass.  TMEM (512 columns): S at [0,128) and [128,256) (alternating key tiles), dP at
+// [256,384) (dS, bf16, is written over the start of each half of dP), dQ accumulator at [384,384+D).
+// Tensor-core order per key tile j:  dQ(j) | dP(j+1) | S(j+2);  element-wise: A(j+1) runs during
+// dQ(j) and dP(j+1), B(j+1) during S(j+2).
 template <int D>
 struct DqSmem {
     static constexpr int kPanels = D / 64;
     static constexpr uint32_t kTileBytes = kTile * D * 2;
-    static constexpr int kStages = 2;
+    static constexpr int kKStages = 3;
+    static constexpr int kVStages = 2;
     static constexpr uint32_t kQ = 0;
     static constexpr uint32_t kDO = kTileBytes;
     static constexpr uint32_t kK = 2 * kTileBytes;
-    static constexpr uint32_t kV = kK + kStages * kTileBytes;
-    static constexpr uint32_t kTotal = kV + kStages * kTileBytes;
+    static constexpr uint32_t kV = kK + kKStages * kTileBytes;
+    static constexpr uint32_t kTotal = kV + kVStages * kTileBytes;
     static constexpr uint32_t kDynamic = kTotal + 1024;
 };
 
@@ -102,9 +127,9 @@ __device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) {
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const __grid_constant__ BwdParams prm) {
     using SM = DqSmem<D>;
-    constexpr int NS = SM::kStages;
-    enum { kBarQ = 0, kBarKFull = 1, kBarKEmpty = 1 + NS, kBarVFull = 1 + 2 * NS, kBarVEmpty = 1 + 3 * NS,
-           kBarSFull = 1 + 4 * NS, kBarDsFull, kBarDqFull, kNumBars };
+    constexpr int NK = SM::kKStages, NV = SM::kVStages;
+    enum { kBarQ = 0, kBarKFull = 1, kBarKEmpty = kBarKFull + NK, kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV,
+           kBarSFull = kBarVEmpty + NV, kBarDpFull = kBarSFull + 2, kBarDsFull, kBarDqFull, kNumBars };
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[kNumBars];
     __shared__ uint32_t tmem_slot;
@@ -125,7 +150,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
     const int n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - t_lo + 1 : 0;
 
     if (tid == 0) {
-        for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), i == kBarDsFull ? 128 : 1);
+        for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), i == kBarDsFull ? kEwWarps : 1);
         fence_mbar_init();
         prefetch_tmap(&prm.tq);
         prefetch_tmap(&prm.tk);
@@ -141,9 +166,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const uint32_t tS = tmem, tDs = tmem, tDp = tmem + 128, tDq = tmem + 256;
+    const uint32_t tS0 = tmem, tDp = tmem + 256, tDq = tmem + 384;
 
     if (warp == 0) {
+        // ---------------- TMA producer ----------------
         if (lane == 0 && n_tiles > 0) {
             mbar_expect_tx(bar(kBarQ), 2 * SM::kTileBytes);
             for (int pnl = 0; pnl < SM::kPanels; ++pnl) {
@@ -151,53 +177,74 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                 tma_load_4d(sDO + pnl * 16384, &prm.tdo, bar(kBarQ), pnl * 64, it.hq, r0, it.b);
             }
             for (int j = 0; j < n_tiles; ++j) {
-                const int s = j % NS, ph = (j / NS) & 1;
+                const int sk = j % NK, sv = j % NV;
                 const int row = (t_lo + j) * kTile;
-                if (!mbar_wait(bar(kBarKEmpty + s), ph ^ 1, 11)) break;
-                mbar_expect_tx(bar(kBarKFull + s), SM::kTileBytes);
+                if (!mbar_wait(bar(kBarKEmpty + sk), ((j / NK) & 1) ^ 1, 11)) break;
+                mbar_expect_tx(bar(kBarKFull + sk), SM::kTileBytes);
                 for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                    tma_load_4d(sK(s) + pnl * 16384, &prm.tk, bar(kBarKFull + s), pnl * 64, it.slot, row, it.b);
-                if (!mbar_wait(bar(kBarVEmpty + s), ph ^ 1, 12)) break;
-                mbar_expect_tx(bar(kBarVFull + s), SM::kTileBytes);
+                    tma_load_4d(sK(sk) + pnl * 16384, &prm.tk, bar(kBarKFull + sk), pnl * 64, it.slot, row, it.b);
+                if (!mbar_wait(bar(kBarVEmpty + sv), ((j / NV) & 1) ^ 1, 12)) break;
+                mbar_expect_tx(bar(kBarVFull + sv), SM::kTileBytes);
                 for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                    tma_load_4d(sV(s) + pnl * 16384, &prm.tv, bar(kBarVFull + s), pnl * 64, it.slot, row, it.b);
+                    tma_load_4d(sV(sv) + pnl * 16384, &prm.tv, bar(kBarVFull + sv), pnl * 64, it.slot, row, it.b);
             }
         }
     } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
         if (lane == 0 && n_tiles > 0) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
-            bool ok = mbar_wait(bar(kBarQ), 0, 13);
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                const int s = j % NS, ph = (j / NS) & 1;
-                ok = mbar_wait(bar(kBarKFull + s), ph, 14) && mbar_wait(bar(kBarVFull + s), ph, 15);
-                if (!ok) break;
+            // S(j) = Q K_j^T into the S buffer j & 1
+            auto issue_s = [&](int j) -> bool {
+                const int sk = j % NK;
+                if (!mbar_wait(bar(kBarKFull + sk), (j / NK) & 1, 14)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-                    mma_ss(tS, make_sdesc(sQ + off, 16, 1024), make_sdesc(sK(s) + off, 16, 1024), idesc_s, k > 0);
+                    mma_ss(tS0 + (j & 1) * 128, make_sdesc(sQ + off, 16, 1024), make_sdesc(sK(sk) + off, 16, 1024), idesc_s,
+                           k > 0);
                 }
+                mma_commit(bar(kBarSFull + (j & 1)));
+                return true;
+            };
+            // dP(j) = dO V_j^T
+            auto issue_dp = [&](int j) -> bool {
+                const int sv = j % NV;
+                if (!mbar_wait(bar(kBarVFull + sv), (j / NV) & 1, 15)) return false;
+                tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-                    mma_ss(tDp, make_sdesc(sDO + off, 16, 1024), make_sdesc(sV(s) + off, 16, 1024), idesc_s, k > 0);
+                    mma_ss(tDp, make_sdesc(sDO + off, 16, 1024), make_sdesc(sV(sv) + off, 16, 1024), idesc_s, k > 0);
                 }
-                mma_commit(bar(kBarVEmpty + s));
-                mma_commit(bar(kBarSFull));
+                mma_commit(bar(kBarVEmpty + sv));
+                mma_commit(bar(kBarDpFull));
+                return true;
+            };
+            bool ok = mbar_wait(bar(kBarQ), 0, 13);
+            ok = ok && issue_s(0) && issue_dp(0);
+            if (ok && n_tiles > 1) ok = issue_s(1);
+            for (int j = 0; ok && j < n_tiles; ++j) {
                 ok = mbar_wait(bar(kBarDsFull), j & 1, 16);
                 if (!ok) break;
                 tc_fence_after();
+                const int sk = j % NK;
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tDq, tDs + k * 8, make_sdesc(sK(s) + k * 2048, 16384, 1024), idesc_dq, (j > 0) || (k > 0));
-                mma_commit(bar(kBarKEmpty + s));
+                    mma_ts(tDq, tDp + packed_a_col(k), make_sdesc(sK(sk) + k * 2048, 16384, 1024), idesc_dq,
+                           (j > 0) || (k > 0));
+                mma_commit(bar(kBarKEmpty + sk));
+                if (j + 1 < n_tiles) ok = issue_dp(j + 1);
+                if (ok && j + 2 < n_tiles) ok = issue_s(j + 2);
             }
             if (ok) mma_commit(bar(kBarDqFull));
         }
-    } else {
-        const int row = 32 * (warp & 3) + lane;
-        const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
+    } else if (warp >= kEwWarp0) {
+        // ---------------- element-wise: thread = query row, 64 of the tile's 128 key columns ----------------
+        const int quarter = warp & 3, half = (warp - kEwWarp0) >> 2;
+        const int row = 32 * quarter + lane;
+        const uint32_t lane_off = (uint32_t)(32 * quarter) << 16;
         const int r = r0 + row;
         const long long p = (long long)geo.q_pos0 + r;
         long long vlo_ll = lo_visible(geo, p, it.flagged) - geo.kv_pos0;
@@ -220,71 +267,86 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
         const uint64_t sl2x2 = f32x2(sl2, sl2);
         const uint64_t nlse2 = f32x2(-lse2, -lse2);
         const uint64_t ndsum2 = f32x2(-dsum, -dsum);
-        // dS = P * (dP - D) for one key tile; MASKED is a compile-time flag so that fully visible
-        // tiles run branch-free straight-line code
-        auto ds_tile = [&](auto masked_c, const int c0) {
+        const uint32_t col_off = (uint32_t)half * 64;
+        float P[64];
+        // phase A: P = 2^(S*scale*log2e - LSE*log2e) for this thread's 64 columns of S buffer `tS`
+        auto phase_a = [&](auto masked_c, const uint32_t tS, const int c0) {
             constexpr bool MASKED = decltype(masked_c)::value;
-            uint32_t sa_[32], sb_[32], da_[32], db_[32];
-            tmem_ld_x32(tS + lane_off, sa_);
-            tmem_ld_x32(tDp + lane_off, da_);
+            uint32_t sa_[32], sb_[32];
+            tmem_ld_x32(tS + lane_off + col_off, sa_);
+            tmem_ld_x32(tS + lane_off + col_off + 32, sb_);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t(&sv)[32] = (c & 1) ? sb_ : sa_;
-                uint32_t(&dv)[32] = (c & 1) ? db_ : da_;
-                uint32_t(&sn)[32] = (c & 1) ? sa_ : sb_;
-                uint32_t(&dn)[32] = (c & 1) ? da_ : db_;
+            for (int c = 0; c < 2; ++c) {
+                uint32_t(&sv)[32] = c ? sb_ : sa_;
                 tmem_wait_ld_dep(sv);
-                tmem_wait_ld_dep(dv);
-                if (c < 3) {
-                    tmem_ld_x32(tS + lane_off + (c + 1) * 32, sn);
-                    tmem_ld_x32(tDp + lane_off + (c + 1) * 32, dn);
-                }
-                uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
                     float t0, t1;
                     f32x2_unpack(fma_f32x2(f32x2_bits(sv[i], sv[i + 1]), sl2x2, nlse2), t0, t1);
-                    const uint64_t p2 = f32x2(ex2(t0), ex2(t1));
-                    const uint64_t ds2 = mul_f32x2(p2, add_f32x2(f32x2_bits(dv[i], dv[i + 1]), ndsum2));
+                    float p0 = ex2(t0), p1 = ex2(t1);
+                    if (MASKED) {
+                        const int col = c0 + (int)col_off + c * 32 + i;
+                        p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
+                        p1 = (col + 1 >= vlo && col + 1 <= vhi) ? p1 : 0.f;
+                    }
+                    P[c * 32 + i] = p0;
+                    P[c * 32 + i + 1] = p1;
+                }
+            }
+        };
+        // phase B: dS = P * (dP - D), rounded to bf16, written over the start of this half of dP
+        auto phase_b = [&]() {
+            uint32_t da_[32], db_[32];
+            tmem_ld_x32(tDp + lane_off + col_off, da_);
+            tmem_ld_x32(tDp + lane_off + col_off + 32, db_);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t(&dv)[32] = c ? db_ : da_;
+                tmem_wait_ld_dep(dv);
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const uint64_t ds2 = mul_f32x2(f32x2(P[c * 32 + i], P[c * 32 + i + 1]),
+                                                   add_f32x2(f32x2_bits(dv[i], dv[i + 1]), ndsum2));
                     float d0, d1;
                     f32x2_unpack(ds2, d0, d1);
-                    if (MASKED) {
-                        const int col = c0 + c * 32 + i;
-                        d0 = (col >= vlo && col <= vhi) ? d0 : 0.f;
-                        d1 = (col + 1 >= vlo && col + 1 <= vhi) ? d1 : 0.f;
-                    }
                     pk[i / 2] = pack_bf16(d0, d1);
                 }
-                tmem_st_x16(tDs + lane_off + c * 16, pk);
+                // both loads have completed before the first store (the wait covers all outstanding loads)
+                tmem_st_x16(tDp + lane_off + col_off + c * 16, pk);
             }
         };
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
             const int c0 = (t_lo + j) * kTile;
             const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), j & 1, 17));
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (j & 1)), (j >> 1) & 1, 17));
             if (!ok) break;
             tc_fence_after();
-            if (masked) ds_tile(std::true_type{}, c0);
-            else ds_tile(std::false_type{}, c0);
+            if (masked) phase_a(std::true_type{}, tS0 + (j & 1) * 128, c0);
+            else phase_a(std::false_type{}, tS0 + (j & 1) * 128, c0);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDpFull), j & 1, 19));
+            if (!ok) break;
+            tc_fence_after();
+            phase_b();
             tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(kBarDsFull));
+            ew_warp_arrive(bar(kBarDsFull), lane);
         }
         if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDqFull), 0, 18));
         tc_fence_after();
+        constexpr int DH = D / 2;  // this thread's share of the row
         __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(prm.dQ) + it.b * prm.q_stride[0] +
-                              (long long)r * prm.q_stride[1] + it.hq * prm.q_stride[2];
+                              (long long)r * prm.q_stride[1] + it.hq * prm.q_stride[2] + half * DH;
         if (n_tiles == 0) {
             if (row_ok)
-                for (int e = 0; e < D; e += 8) *reinterpret_cast<uint4*>(grow + e) = make_uint4(0, 0, 0, 0);
+                for (int e = 0; e < DH; e += 8) *reinterpret_cast<uint4*>(grow + e) = make_uint4(0, 0, 0, 0);
         } else if (ok) {
             const float sc = prm.sm_scale;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < DH / 32; ++c) {
                 uint32_t v[32];
-                tmem_ld_x32(tDq + lane_off + c * 32, v);
-                tmem_wait_ld();
+                tmem_ld_x32(tDq + lane_off + half * DH + c * 32, v);
+                tmem_wait_ld_dep(v);
                 if (row_ok) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
@@ -314,8 +376,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
 // segment from the diagonal on, plus the whole next segment when the tile reaches into the last
 // T positions (the carried tail).  The loop set does not depend on the head flag.
 // Transposed products keep the key on the accumulator row: S^T = K Q^T, dP^T = V dO^T,
-// dV += P^T dO, dK += dS^T Q.  TMEM (512 columns): S^T / P^T at [0,128), dP^T / dS^T at [128,256)
-// (the bf16 forms alias the first 64 columns of each), dV at [256,256+D), dK at [384,384+D).
+// dV += P^T dO, dK += dS^T Q.  TMEM (512 columns): S^T at [0,128), dP^T at [128,256) (P^T and dS^T,
+// bf16, are written over the start of each half of S^T and dP^T), dV at [256,256+D), dK at [384,384+D).
+// Tensor-core order per (head, query tile) i:  dV(i) | S^T(i+1) | dK(i) | dP^T(i+1);  element-wise:
+// B(i) runs during dV(i) and S^T(i+1), A(i+1) during dK(i) and dP^T(i+1).
 template <int D>
 struct DkvSmem {
     static constexpr int kPanels = D / 64;
@@ -329,13 +393,13 @@ struct DkvSmem {
     static constexpr uint32_t kDynamic = kTotal + 1024;
 };
 
-__device__ __forceinline__ void compute_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const __grid_constant__ BwdParams prm) {
     using SM = DkvSmem<D>;
     constexpr int NS = SM::kStages;
-    enum { kBarKV = 0, kBarQFull = 1, kBarQEmpty = 1 + NS, kBarSFull = 1 + 2 * NS, kBarPFull, kBarDone, kNumBars };
+    enum { kBarKV = 0, kBarQFull = 1, kBarQEmpty = kBarQFull + NS, kBarDoFull = kBarQEmpty + NS,
+           kBarDoEmpty = kBarDoFull + NS, kBarSFull = kBarDoEmpty + NS, kBarDpFull, kBarPFull, kBarDsFull, kBarDone,
+           kNumBars };
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[kNumBars];
     __shared__ uint32_t tmem_slot;
@@ -363,7 +427,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
     const int n_it = n_qt * prm.g;
 
     if (tid == 0) {
-        for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), i == kBarPFull ? 128 : 1);
+        for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i == kBarPFull || i == kBarDsFull) ? kEwWarps : 1);
         fence_mbar_init();
         prefetch_tmap(&prm.tq);
         prefetch_tmap(&prm.tk);
@@ -379,9 +443,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const uint32_t tSt = tmem, tPt = tmem, tDpt = tmem + 128, tDst = tmem + 128, tDv = tmem + 256, tDk = tmem + 384;
+    const uint32_t tSt = tmem, tDpt = tmem + 128, tDv = tmem + 256, tDk = tmem + 384;
 
     if (warp == 0) {
+        // ---------------- TMA producer ----------------
         if (lane == 0 && n_it > 0) {
             mbar_expect_tx(bar(kBarKV), 2 * SM::kTileBytes);
             for (int pnl = 0; pnl < SM::kPanels; ++pnl) {
@@ -393,51 +458,77 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
                 const int hq = hq0 + i / n_qt;
                 const int row = (qt_lo + i % n_qt) * kTile;
                 if (!mbar_wait(bar(kBarQEmpty + s), ph ^ 1, 21)) break;
-                mbar_expect_tx(bar(kBarQFull + s), 2 * SM::kTileBytes);
-                for (int pnl = 0; pnl < SM::kPanels; ++pnl) {
+                mbar_expect_tx(bar(kBarQFull + s), SM::kTileBytes);
+                for (int pnl = 0; pnl < SM::kPanels; ++pnl)
                     tma_load_4d(sQ(s) + pnl * 16384, &prm.tq, bar(kBarQFull + s), pnl * 64, hq, row, b);
-                    tma_load_4d(sDO(s) + pnl * 16384, &prm.tdo, bar(kBarQFull + s), pnl * 64, hq, row, b);
-                }
+                if (!mbar_wait(bar(kBarDoEmpty + s), ph ^ 1, 27)) break;
+                mbar_expect_tx(bar(kBarDoFull + s), SM::kTileBytes);
+                for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                    tma_load_4d(sDO(s) + pnl * 16384, &prm.tdo, bar(kBarDoFull + s), pnl * 64, hq, row, b);
             }
         }
     } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
         if (lane == 0 && n_it > 0) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_g = make_idesc_bf16(128, D, 0, 1);
-            bool ok = mbar_wait(bar(kBarKV), 0, 22);
-            for (int i = 0; ok && i < n_it; ++i) {
-                const int s = i % NS, ph = (i / NS) & 1;
-                ok = mbar_wait(bar(kBarQFull + s), ph, 23);
-                if (!ok) break;
+            auto issue_st = [&](int i) -> bool {   // S^T(i) = K Q_i^T
+                const int s = i % NS;
+                if (!mbar_wait(bar(kBarQFull + s), (i / NS) & 1, 23)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
                     mma_ss(tSt, make_sdesc(sKt + off, 16, 1024), make_sdesc(sQ(s) + off, 16, 1024), idesc_s, k > 0);
                 }
+                mma_commit(bar(kBarSFull));
+                return true;
+            };
+            auto issue_dpt = [&](int i) -> bool {  // dP^T(i) = V dO_i^T
+                const int s = i % NS;
+                if (!mbar_wait(bar(kBarDoFull + s), (i / NS) & 1, 28)) return false;
+                tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
                     mma_ss(tDpt, make_sdesc(sVt + off, 16, 1024), make_sdesc(sDO(s) + off, 16, 1024), idesc_s, k > 0);
                 }
-                mma_commit(bar(kBarSFull));
+                mma_commit(bar(kBarDpFull));
+                return true;
+            };
+            bool ok = mbar_wait(bar(kBarKV), 0, 22);
+            ok = ok && issue_st(0) && issue_dpt(0);
+            for (int i = 0; ok && i < n_it; ++i) {
+                const int s = i % NS;
                 ok = mbar_wait(bar(kBarPFull), i & 1, 24);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tDv, tPt + k * 8, make_sdesc(sDO(s) + k * 2048, 16384, 1024), idesc_g, (i > 0) || (k > 0));
+                    mma_ts(tDv, tSt + packed_a_col(k), make_sdesc(sDO(s) + k * 2048, 16384, 1024), idesc_g,
+                           (i > 0) || (k > 0));
+                mma_commit(bar(kBarDoEmpty + s));
+                if (i + 1 < n_it) ok = issue_st(i + 1);
+                if (!ok) break;
+                ok = mbar_wait(bar(kBarDsFull), i & 1, 29);
+                if (!ok) break;
+                tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tDk, tDst + k * 8, make_sdesc(sQ(s) + k * 2048, 16384, 1024), idesc_g, (i > 0) || (k > 0));
+                    mma_ts(tDk, tDpt + packed_a_col(k), make_sdesc(sQ(s) + k * 2048, 16384, 1024), idesc_g,
+                           (i > 0) || (k > 0));
                 mma_commit(bar(kBarQEmpty + s));
+                if (i + 1 < n_it) ok = issue_dpt(i + 1);
             }
             if (ok) mma_commit(bar(kBarDone));
         }
-    } else {
-        const int ctid = tid - 64;  // 0..127 among the compute warps
-        const int row = 32 * (warp & 3) + lane;  // key row of this thread inside the tile
-        const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
+    } else if (warp >= kEwWarp0) {
+        // ---------------- element-wise: thread = key row, 64 of the tile's 128 query columns ----------------
+        const int quarter = warp & 3, half = (warp - kEwWarp0) >> 2;
+        const int ctid = tid - kEwWarp0 * 32;      // 0..255 among the element-wise threads
+        const int row = 32 * quarter + lane;       // key row of this thread inside the tile
+        const uint32_t lane_off = (uint32_t)(32 * quarter) << 16;
+        const uint32_t col_off = (uint32_t)half * 64;
         const int jl = c0 + row;
         const long long jpos = (long long)geo.kv_pos0 + jl;
         // query rows that read this key differentiably: [qlo, qhi]
@@ -454,112 +545,127 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
         const bool keys_in_range = c0 + kTile <= geo.kv_len && jfirst >= 0;
 
         const float sl2 = prm.scale_log2;
-        auto stat_index = [&](int i) {
+        // threads 0..127 stage LSE*log2e of the item's query rows, threads 128..255 the row dots D
+        auto fetch_stat = [&](int i) -> float {
             const int hq = hq0 + i / n_qt;
-            const int qr = (qt_lo + i % n_qt) * kTile + ctid;
-            return qr < geo.Lq ? ((long long)b * prm.Hq + hq) * geo.Lq + qr : -1ll;
-        };
-        float lse_next = INFINITY, d_next = 0.f;
-        if (n_it > 0) {
-            const long long si = stat_index(0);
-            if (si >= 0) {
+            const int qr = (qt_lo + i % n_qt) * kTile + (ctid & 127);
+            if (qr >= geo.Lq) return ctid < 128 ? INFINITY : 0.f;
+            const long long si = ((long long)b * prm.Hq + hq) * geo.Lq + qr;
+            if (ctid < 128) {
                 const float l = prm.LSE[si];
-                lse_next = (l == -INFINITY) ? INFINITY : l * kLog2e;
-                d_next = prm.Dvec[si];
+                return (l == -INFINITY) ? INFINITY : l * kLog2e;
             }
-        }
+            return prm.Dvec[si];
+        };
+        float stat_next = n_it > 0 ? fetch_stat(0) : 0.f;
         const uint64_t sl2x2 = f32x2(sl2, sl2);
-        // P^T = 2^(S^T*scale*log2e - LSE_q*log2e) and dS^T = P^T * (dP^T - D_q) for one query tile
-        // (query = column); MASKED is a compile-time flag so that full tiles run branch-free code
-        auto pt_tile = [&](auto masked_c, const int buf, const int q0) {
+        float P[64];
+        // phase A: P^T = 2^(S^T*scale*log2e - LSE_q*log2e) (query = column), bf16 copy over the start of
+        // this half of S^T
+        auto phase_a = [&](auto masked_c, const int buf, const int q0) {
             constexpr bool MASKED = decltype(masked_c)::value;
-            uint32_t sa_[32], sb_[32], da_[32], db_[32];
-            tmem_ld_x32(tSt + lane_off, sa_);
-            tmem_ld_x32(tDpt + lane_off, da_);
+            uint32_t sa_[32], sb_[32];
+            tmem_ld_x32(tSt + lane_off + col_off, sa_);
+            tmem_ld_x32(tSt + lane_off + col_off + 32, sb_);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t(&sv)[32] = (c & 1) ? sb_ : sa_;
-                uint32_t(&dv)[32] = (c & 1) ? db_ : da_;
-                uint32_t(&sn)[32] = (c & 1) ? sa_ : sb_;
-                uint32_t(&dn)[32] = (c & 1) ? da_ : db_;
+            for (int c = 0; c < 2; ++c) {
+                uint32_t(&sv)[32] = c ? sb_ : sa_;
                 tmem_wait_ld_dep(sv);
-                tmem_wait_ld_dep(dv);
-                if (c < 3) {
-                    tmem_ld_x32(tSt + lane_off + (c + 1) * 32, sn);
-                    tmem_ld_x32(tDpt + lane_off + (c + 1) * 32, dn);
-                }
-                uint32_t pk[16], dk[16];
+                uint32_t pk[16];
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    const float2 l2 = *reinterpret_cast<const float2*>(&s_lse[buf][c * 32 + e]);
-                    const float2 dd = *reinterpret_cast<const float2*>(&s_dsum[buf][c * 32 + e]);
-                    float t0, t1;
-                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[e], sv[e + 1]), sl2x2, f32x2(-l2.x, -l2.y)), t0, t1);
-                    float p0 = ex2(t0), p1 = ex2(t1);
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[buf][col_off + c * 32 + e]);
+                    float t0, t1, t2, t3;
+                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[e], sv[e + 1]), sl2x2, f32x2(-l4.x, -l4.y)), t0, t1);
+                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[e + 2], sv[e + 3]), sl2x2, f32x2(-l4.z, -l4.w)), t2, t3);
+                    float p0 = ex2(t0), p1 = ex2(t1), p2 = ex2(t2), p3 = ex2(t3);
                     if (MASKED) {
-                        const int q = q0 + c * 32 + e;
+                        const int q = q0 + (int)col_off + c * 32 + e;
                         p0 = (q >= qlo && q <= qhi) ? p0 : 0.f;
                         p1 = (q + 1 >= qlo && q + 1 <= qhi) ? p1 : 0.f;
+                        p2 = (q + 2 >= qlo && q + 2 <= qhi) ? p2 : 0.f;
+                        p3 = (q + 3 >= qlo && q + 3 <= qhi) ? p3 : 0.f;
                     }
-                    const uint64_t ds2 = mul_f32x2(f32x2(p0, p1), add_f32x2(f32x2_bits(dv[e], dv[e + 1]), f32x2(-dd.x, -dd.y)));
-                    float d0, d1;
-                    f32x2_unpack(ds2, d0, d1);
+                    P[c * 32 + e] = p0;
+                    P[c * 32 + e + 1] = p1;
+                    P[c * 32 + e + 2] = p2;
+                    P[c * 32 + e + 3] = p3;
                     pk[e / 2] = pack_bf16(p0, p1);
-                    dk[e / 2] = pack_bf16(d0, d1);
+                    pk[e / 2 + 1] = pack_bf16(p2, p3);
                 }
-                tmem_st_x16(tPt + lane_off + c * 16, pk);
-                tmem_st_x16(tDst + lane_off + c * 16, dk);
+                tmem_st_x16(tSt + lane_off + col_off + c * 16, pk);
+            }
+        };
+        // phase B: dS^T = P^T * (dP^T - D_q), bf16, over the start of this half of dP^T
+        auto phase_b = [&](const int buf) {
+            uint32_t da_[32], db_[32];
+            tmem_ld_x32(tDpt + lane_off + col_off, da_);
+            tmem_ld_x32(tDpt + lane_off + col_off + 32, db_);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t(&dv)[32] = c ? db_ : da_;
+                tmem_wait_ld_dep(dv);
+                uint32_t dk[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float4 d4 = *reinterpret_cast<const float4*>(&s_dsum[buf][col_off + c * 32 + e]);
+                    float d0, d1, d2, d3;
+                    f32x2_unpack(mul_f32x2(f32x2(P[c * 32 + e], P[c * 32 + e + 1]),
+                                           add_f32x2(f32x2_bits(dv[e], dv[e + 1]), f32x2(-d4.x, -d4.y))), d0, d1);
+                    f32x2_unpack(mul_f32x2(f32x2(P[c * 32 + e + 2], P[c * 32 + e + 3]),
+                                           add_f32x2(f32x2_bits(dv[e + 2], dv[e + 3]), f32x2(-d4.z, -d4.w))), d2, d3);
+                    dk[e / 2] = pack_bf16(d0, d1);
+                    dk[e / 2 + 1] = pack_bf16(d2, d3);
+                }
+                tmem_st_x16(tDpt + lane_off + col_off + c * 16, dk);
             }
         };
         bool ok = true;
         for (int i = 0; i < n_it; ++i) {
             const int buf = i & 1;
-            s_lse[buf][ctid] = lse_next;
-            s_dsum[buf][ctid] = d_next;
-            compute_bar_sync();
-            lse_next = INFINITY;
-            d_next = 0.f;
-            if (i + 1 < n_it) {
-                const long long si = stat_index(i + 1);
-                if (si >= 0) {
-                    const float l = prm.LSE[si];
-                    lse_next = (l == -INFINITY) ? INFINITY : l * kLog2e;
-                    d_next = prm.Dvec[si];
-                }
-            }
+            if (ctid < 128) s_lse[buf][ctid] = stat_next;
+            else s_dsum[buf][ctid - 128] = stat_next;
+            ew_bar_sync();
+            if (i + 1 < n_it) stat_next = fetch_stat(i + 1);
             const int q0 = (qt_lo + i % n_qt) * kTile;
             const bool masked = !(keys_in_range && q0 >= full_qlo && q0 + kTile - 1 <= full_qhi);
-            // after a failed wait keep looping (without touching TMEM) so that every compute thread
+            // after a failed wait keep looping (without touching TMEM) so that every element-wise thread
             // still reaches the named barrier above the same number of times
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), i & 1, 25));
             if (!ok) continue;
             tc_fence_after();
-            if (masked) pt_tile(std::true_type{}, buf, q0);
-            else pt_tile(std::false_type{}, buf, q0);
+            if (masked) phase_a(std::true_type{}, buf, q0);
+            else phase_a(std::false_type{}, buf, q0);
             tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(kBarPFull));
+            ew_warp_arrive(bar(kBarPFull), lane);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDpFull), i & 1, 30));
+            if (!ok) continue;
+            tc_fence_after();
+            phase_b(buf);
+            tmem_wait_st();
+            ew_warp_arrive(bar(kBarDsFull), lane);
         }
         if (n_it > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDone), 0, 26));
         tc_fence_after();
+        constexpr int DH = D / 2;
         const bool row_ok = jl < geo.kv_len;
         __nv_bfloat16* gk = reinterpret_cast<__nv_bfloat16*>(prm.dK) + b * prm.k_stride[0] +
-                            (long long)jl * prm.k_stride[1] + slot * prm.k_stride[2];
+                            (long long)jl * prm.k_stride[1] + slot * prm.k_stride[2] + half * DH;
         __nv_bfloat16* gv = reinterpret_cast<__nv_bfloat16*>(prm.dV) + b * prm.v_stride[0] +
-                            (long long)jl * prm.v_stride[1] + slot * prm.v_stride[2];
+                            (long long)jl * prm.v_stride[1] + slot * prm.v_stride[2] + half * DH;
         if (n_it == 0) {
             if (row_ok)
-                for (int e = 0; e < D; e += 8) {
+                for (int e = 0; e < DH; e += 8) {
                     *reinterpret_cast<uint4*>(gk + e) = make_uint4(0, 0, 0, 0);
                     *reinterpret_cast<uint4*>(gv + e) = make_uint4(0, 0, 0, 0);
                 }
         } else if (ok) {
             const float sc = prm.sm_scale;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < DH / 32; ++c) {
                 uint32_t v[32], k[32];
-                tmem_ld_x32(tDv + lane_off + c * 32, v);
-                tmem_ld_x32(tDk + lane_off + c * 32, k);
+                tmem_ld_x32(tDv + lane_off + half * DH + c * 32, v);
+                tmem_ld_x32(tDk + lane_off + half * DH + c * 32, k);
                 tmem_wait_ld();
                 if (row_ok) {
 #pragma unroll
