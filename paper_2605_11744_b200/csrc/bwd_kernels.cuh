@@ -74,10 +74,10 @@ __device__ __forceinline__ void ew_bar_sync() { asm volatile("bar.sync 1, 256;" 
 __device__ __forceinline__ uint32_t packed_a_col(int k) { return (uint32_t)((k >> 2) * 64 + (k & 3) * 8); }
 
 // ------------------------------------------------------------------------------------------
-// dQ pass.  TMEM (512 columns): S at [0,128) and [128,256) (alternating key tiles), dP at
-// [256,384) (dS, bf16, is written over the start of each half of dP), dQ accumulator at [384,384+D).
-// Tensor-core order per key tile j:  dQ(j) | dP(j+1) | S(j+2);  element-wise: A(j+1) runs during
-// dQ(j) and dP(j+1), B(j+1) during S(j+2).
+// dQ pass.  TMEM (512 columns): S at [0,128) and [128,256) (alternating key tiles; dS, bf16, is
+// written over the start of each half of the tile's S buffer), dP at [256,384), dQ accumulator at
+// [384,384+D).  Tensor-core order per key tile j, one straight run once dS(j) is there:
+// dP(j+1) | dQ(j) | S(j+2);  element-wise: A(j+1) runs meanwhile, B(j+1) as soon as dP(j+1) is done.
 template <int D>
 struct DqSmem {
     static constexpr int kPanels = D / 64;
@@ -127,6 +127,8 @@ __device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) {
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const __grid_constant__ BwdParams prm) {
     using SM = DqSmem<D>;
+    constexpr int trace_id = 1;
+    (void)trace_id;
     constexpr int NK = SM::kKStages, NV = SM::kVStages;
     enum { kBarQ = 0, kBarKFull = 1, kBarKEmpty = kBarKFull + NK, kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV,
            kBarSFull = kBarVEmpty + NV, kBarDpFull = kBarSFull + 2, kBarDsFull, kBarDqFull, kNumBars };
@@ -190,15 +192,16 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0 && n_tiles > 0) {
+        // ---------------- MMA issuer (whole warp, uniform control flow; one elected lane issues) ----------------
+        if (n_tiles > 0) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
-            // S(j) = Q K_j^T into the S buffer j & 1
-            auto issue_s = [&](int j) -> bool {
+            // Waits on tiles brought by TMA need no tcgen05 fence; they are taken ahead of the wait on the
+            // element-wise warps so that the products of one key tile go out as one straight run of MMAs.
+            auto wait_k = [&](int j) { return warp_wait(bar(kBarKFull + j % NK), (j / NK) & 1, 14); };
+            auto wait_v = [&](int j) { return warp_wait(bar(kBarVFull + j % NV), (j / NV) & 1, 15); };
+            auto issue_s = [&](int j) {   // S(j) = Q K_j^T into the S buffer j & 1
                 const int sk = j % NK;
-                if (!mbar_wait(bar(kBarKFull + sk), (j / NK) & 1, 14)) return false;
-                tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
@@ -206,13 +209,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                            k > 0);
                 }
                 mma_commit(bar(kBarSFull + (j & 1)));
-                return true;
             };
-            // dP(j) = dO V_j^T
-            auto issue_dp = [&](int j) -> bool {
+            auto issue_dp = [&](int j) {  // dP(j) = dO V_j^T
                 const int sv = j % NV;
-                if (!mbar_wait(bar(kBarVFull + sv), (j / NV) & 1, 15)) return false;
-                tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
@@ -220,23 +219,32 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                 }
                 mma_commit(bar(kBarVEmpty + sv));
                 mma_commit(bar(kBarDpFull));
-                return true;
             };
-            bool ok = mbar_wait(bar(kBarQ), 0, 13);
-            ok = ok && issue_s(0) && issue_dp(0);
-            if (ok && n_tiles > 1) ok = issue_s(1);
+            bool ok = warp_wait(bar(kBarQ), 0, 13) && wait_k(0) && wait_v(0);
+            if (ok) {
+                issue_s(0);
+                issue_dp(0);
+            }
+            if (ok && n_tiles > 1 && (ok = wait_k(1))) issue_s(1);
             for (int j = 0; ok && j < n_tiles; ++j) {
-                ok = mbar_wait(bar(kBarDsFull), j & 1, 16);
+                if (j + 1 < n_tiles) ok = wait_v(j + 1);
+                ok = ok && warp_wait(bar(kBarDsFull), j & 1, 16);   // dS(j) written, dP(j) read
                 if (!ok) break;
                 tc_fence_after();
+                TRACE(lane == 0, j * 16 + 4);
+                if (j + 1 < n_tiles) issue_dp(j + 1);   // first: phase B of the next tile waits for it
+                TRACE(lane == 0, j * 16 + 6);
                 const int sk = j % NK;
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tDq, tDp + packed_a_col(k), make_sdesc(sK(sk) + k * 2048, 16384, 1024), idesc_dq,
+                    mma_ts(tDq, tS0 + (j & 1) * 128 + packed_a_col(k), make_sdesc(sK(sk) + k * 2048, 16384, 1024), idesc_dq,
                            (j > 0) || (k > 0));
                 mma_commit(bar(kBarKEmpty + sk));
-                if (j + 1 < n_tiles) ok = issue_dp(j + 1);
-                if (ok && j + 2 < n_tiles) ok = issue_s(j + 2);
+                TRACE(lane == 0, j * 16 + 7);
+                // K(j+2) reuses the stage dQ(j-1) released one run ago: its load gets the first two products
+                // of this run as extra time before it is waited for
+                if (j + 2 < n_tiles && (ok = wait_k(j + 2))) issue_s(j + 2);    // overwrites dS(j): after dQ(j)
+                TRACE(lane == 0, j * 16 + 5);
             }
             if (ok) mma_commit(bar(kBarDqFull));
         }
@@ -294,8 +302,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                 }
             }
         };
-        // phase B: dS = P * (dP - D), rounded to bf16, written over the start of this half of dP
-        auto phase_b = [&]() {
+        // phase B: dS = P * (dP - D), rounded to bf16, written over the start of this half of the tile's S
+        // buffer (its scores went into P in phase A; the next product into that buffer is issued after dQ)
+        auto phase_b = [&](const uint32_t tS) {
             uint32_t da_[32], db_[32];
             tmem_ld_x32(tDp + lane_off + col_off, da_);
             tmem_ld_x32(tDp + lane_off + col_off + 32, db_);
@@ -312,8 +321,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                     f32x2_unpack(ds2, d0, d1);
                     pk[i / 2] = pack_bf16(d0, d1);
                 }
-                // both loads have completed before the first store (the wait covers all outstanding loads)
-                tmem_st_x16(tDp + lane_off + col_off + c * 16, pk);
+                tmem_st_x16(tS + lane_off + col_off + c * 16, pk);
             }
         };
         bool ok = true;
@@ -323,14 +331,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
             ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (j & 1)), (j >> 1) & 1, 17));
             if (!ok) break;
             tc_fence_after();
+            TRACE(tid == 128, j * 16 + 0);
             if (masked) phase_a(std::true_type{}, tS0 + (j & 1) * 128, c0);
             else phase_a(std::false_type{}, tS0 + (j & 1) * 128, c0);
+            TRACE(tid == 128, j * 16 + 1);
             ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDpFull), j & 1, 19));
             if (!ok) break;
             tc_fence_after();
-            phase_b();
+            TRACE(tid == 128, j * 16 + 2);
+            phase_b(tS0 + (j & 1) * 128);
             tmem_wait_st();
             ew_warp_arrive(bar(kBarDsFull), lane);
+            TRACE(tid == 128, j * 16 + 3);
+            TRACE(lane == 0, j * 16 + 8 + (warp - kEwWarp0));
         }
         if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDqFull), 0, 18));
         tc_fence_after();
@@ -396,6 +409,8 @@ struct DkvSmem {
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const __grid_constant__ BwdParams prm) {
     using SM = DkvSmem<D>;
+    constexpr int trace_id = 2;
+    (void)trace_id;
     constexpr int NS = SM::kStages;
     enum { kBarKV = 0, kBarQFull = 1, kBarQEmpty = kBarQFull + NS, kBarDoFull = kBarQEmpty + NS,
            kBarDoEmpty = kBarDoFull + NS, kBarSFull = kBarDoEmpty + NS, kBarDpFull, kBarPFull, kBarDsFull, kBarDone,
@@ -468,13 +483,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0 && n_it > 0) {
+        // ---------------- MMA issuer (whole warp, uniform control flow; one elected lane issues) ----------------
+        if (n_it > 0) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_g = make_idesc_bf16(128, D, 0, 1);
             auto issue_st = [&](int i) -> bool {   // S^T(i) = K Q_i^T
                 const int s = i % NS;
-                if (!mbar_wait(bar(kBarQFull + s), (i / NS) & 1, 23)) return false;
+                if (!warp_wait(bar(kBarQFull + s), (i / NS) & 1, 23)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
@@ -486,7 +501,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
             };
             auto issue_dpt = [&](int i) -> bool {  // dP^T(i) = V dO_i^T
                 const int s = i % NS;
-                if (!mbar_wait(bar(kBarDoFull + s), (i / NS) & 1, 28)) return false;
+                if (!warp_wait(bar(kBarDoFull + s), (i / NS) & 1, 28)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
@@ -496,13 +511,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
                 mma_commit(bar(kBarDpFull));
                 return true;
             };
-            bool ok = mbar_wait(bar(kBarKV), 0, 22);
+            bool ok = warp_wait(bar(kBarKV), 0, 22);
             ok = ok && issue_st(0) && issue_dpt(0);
             for (int i = 0; ok && i < n_it; ++i) {
                 const int s = i % NS;
-                ok = mbar_wait(bar(kBarPFull), i & 1, 24);
+                ok = warp_wait(bar(kBarPFull), i & 1, 24);
                 if (!ok) break;
                 tc_fence_after();
+                TRACE(lane == 0, i * 8 + 4);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
                     mma_ts(tDv, tSt + packed_a_col(k), make_sdesc(sDO(s) + k * 2048, 16384, 1024), idesc_g,
@@ -510,15 +526,18 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
                 mma_commit(bar(kBarDoEmpty + s));
                 if (i + 1 < n_it) ok = issue_st(i + 1);
                 if (!ok) break;
-                ok = mbar_wait(bar(kBarDsFull), i & 1, 29);
+                TRACE(lane == 0, i * 8 + 5);
+                ok = warp_wait(bar(kBarDsFull), i & 1, 29);
                 if (!ok) break;
                 tc_fence_after();
+                TRACE(lane == 0, i * 8 + 6);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
                     mma_ts(tDk, tDpt + packed_a_col(k), make_sdesc(sQ(s) + k * 2048, 16384, 1024), idesc_g,
                            (i > 0) || (k > 0));
                 mma_commit(bar(kBarQEmpty + s));
                 if (i + 1 < n_it) ok = issue_dpt(i + 1);
+                TRACE(lane == 0, i * 8 + 7);
             }
             if (ok) mma_commit(bar(kBarDone));
         }
@@ -634,16 +653,20 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), i & 1, 25));
             if (!ok) continue;
             tc_fence_after();
+            TRACE(tid == 128, i * 8 + 0);
             if (masked) phase_a(std::true_type{}, buf, q0);
             else phase_a(std::false_type{}, buf, q0);
             tmem_wait_st();
             ew_warp_arrive(bar(kBarPFull), lane);
+            TRACE(tid == 128, i * 8 + 1);
             ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDpFull), i & 1, 30));
             if (!ok) continue;
             tc_fence_after();
+            TRACE(tid == 128, i * 8 + 2);
             phase_b(buf);
             tmem_wait_st();
             ew_warp_arrive(bar(kBarDsFull), lane);
+            TRACE(tid == 128, i * 8 + 3);
         }
         if (n_it > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDone), 0, 26));
         tc_fence_after();

@@ -67,6 +67,8 @@ __device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) {
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __grid_constant__ FwdParams prm) {
     using SM = FwdSmem<D>;
+    constexpr int trace_id = 0;
+    (void)trace_id;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[kFwdBars];
     __shared__ uint32_t tmem_slot;
@@ -130,8 +132,8 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0 && n_tiles > 0) {
+        // ---------------- MMA issuer (whole warp, uniform control flow; one elected lane issues) ----------------
+        if (n_tiles > 0) {
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
             auto issue_qk = [&]() {
@@ -141,7 +143,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
                     mma_ss(tS, make_sdesc(sQ + off, 16, 1024), make_sdesc(sK + off, 16, 1024), idesc_qk, k > 0);
                 }
             };
-            bool ok = mbar_wait(bar(kBarQ), 0, 3) && mbar_wait(bar(kBarKFull), 0, 4);
+            bool ok = warp_wait(bar(kBarQ), 0, 3) && warp_wait(bar(kBarKFull), 0, 4);
             if (ok) {
                 tc_fence_after();
                 issue_qk();
@@ -149,22 +151,22 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
                 mma_commit(bar(kBarSFull));
             }
             for (int j = 0; ok && j < n_tiles; ++j) {
-                ok = mbar_wait(bar(kBarPFull), j & 1, 5) && mbar_wait(bar(kBarVFull), j & 1, 6);
+                ok = warp_wait(bar(kBarPFull), j & 1, 5) && warp_wait(bar(kBarVFull), j & 1, 6);
                 if (!ok) break;
                 tc_fence_after();
-                TRACE(true, j * 8 + 4);
+                TRACE(lane == 0, j * 8 + 4);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
                     mma_ts(tO, tP + k * 8, make_sdesc(sV + k * 2048, 16384, 1024), idesc_pv, (j > 0) || (k > 0));
                 mma_commit(bar(kBarVEmpty));
-                TRACE(true, j * 8 + 5);
+                TRACE(lane == 0, j * 8 + 5);
                 if (j + 1 < n_tiles) {
-                    ok = mbar_wait(bar(kBarKFull), (j + 1) & 1, 7);
+                    ok = warp_wait(bar(kBarKFull), (j + 1) & 1, 7);
                     if (!ok) break;
                     tc_fence_after();
-                    TRACE(true, j * 8 + 6);
+                    TRACE(lane == 0, j * 8 + 6);
                     issue_qk();
-                    TRACE(true, j * 8 + 7);
+                    TRACE(lane == 0, j * 8 + 7);
                     mma_commit(bar(kBarKEmpty));
                     mma_commit(bar(kBarSFull));
                 } else {

@@ -13,10 +13,12 @@ namespace segattn {
 __device__ int g_device_status = 0;
 
 #ifdef SEGATTN_TRACE
-// Debug-only timeline: TRACE(slot) stores clock64 of one chosen CTA into a global buffer.
+// Debug-only timeline: TRACE(slot) stores clock64 of one chosen CTA of one chosen kernel (the
+// kernel's `trace_id`) into a global buffer.
 __device__ long long g_trace[4096];
 __device__ int g_trace_block = 0;
-#define TRACE(cond, idx) do { if ((cond) && blockIdx.x == g_trace_block && (idx) < 4096) { long long t_; asm volatile("mov.u64 %0, %clock64;" : "=l"(t_)); g_trace[(idx)] = t_; } } while (0)
+__device__ int g_trace_kernel = 0;
+#define TRACE(cond, idx) do { if ((cond) && blockIdx.x == g_trace_block && g_trace_kernel == trace_id && (idx) < 4096) { long long t_; asm volatile("mov.u64 %0, %clock64;" : "=l"(t_)); g_trace[(idx)] = t_; } } while (0)
 #else
 #define TRACE(cond, idx) do { } while (0)
 #endif
@@ -190,12 +192,16 @@ __device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_byte
     return uint64_t((saddr & 0x3FFFFu) >> 4) | (uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16) |
            (uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
 }
+// The three issue functions below are WARP-COLLECTIVE: all 32 lanes of a converged warp call them
+// with the same arguments and one elected lane (the same one every time) issues the instruction.
+// Keeping the issuing warp's control flow uniform matters: a lone lane inside a divergent branch
+// issues several times slower when other warps keep the scheduler busy.
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "{\n\t.reg .pred p, q;\n\telect.sync _|q, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -203,14 +209,21 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "{\n\t.reg .pred p, q;\n\telect.sync _|q, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// Arrive once on `bar` when every MMA this thread issued so far has finished.
+// Arrive once on `bar` when every MMA the elected lane issued so far has finished.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
+        : "memory");
+}
+// A bounded wait executed by a whole warp, with a warp-uniform result.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, int site) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, site));
 }
 
 // ---- small numeric helpers ---------------------------------------------------------------------

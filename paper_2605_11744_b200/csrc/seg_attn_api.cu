@@ -341,6 +341,9 @@ extern "C" segattn_status seg_attn_bwd_static(const seg_attn_params* p, const vo
 extern "C" int seg_attn_debug_trace(long long* out, int n, int set_block) {
     if (set_block >= 0) {
         static long long zeros[4096];
+        const int kernel_id = set_block >> 24;  // 0 forward, 1 dQ pass, 2 dK/dV pass
+        set_block &= 0xffffff;
+        cudaMemcpyToSymbol(g_trace_kernel, &kernel_id, sizeof(int));
         cudaMemcpyToSymbol(g_trace_block, &set_block, sizeof(int));
         cudaMemcpyToSymbol(g_trace, zeros, sizeof(zeros));
         return 0;
