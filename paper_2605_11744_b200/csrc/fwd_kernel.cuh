@@ -1,11 +1,18 @@
-// Forward kernel: O = softmax(Q K^T * scale + mask) V and LSE for one 128-row query tile of one
-// (batch, query head) per CTA (Appendix C, Eqs. "attn" and "ctx"), visiting only the key tiles
-// the segment / tail / past-access mask leaves visible.
+// Forward kernel: O = softmax(Q K^T * scale + mask) V and LSE (Appendix C, Eqs. "attn" and "ctx"),
+// visiting only the key tiles the segment / tail / past-access mask leaves visible.
 //
-// Roles (192 threads): warp 0 = TMA producer, warp 1 = tcgen05 MMA issuer and TMEM owner,
-// warps 2..5 = softmax + epilogue (thread <-> query row through the 32x32b TMEM shape).
-// TMEM (256 columns): S / P at columns [0,128) (P, bf16, aliases the first 64), O at [128,128+D).
-// Two CTAs are resident per SM so that one CTA's softmax overlaps the other's MMAs.
+// Persistent: one CTA per SM walks a static list of work items (one 128-row query tile of one
+// (batch, query head) each), heaviest items first, dealt round-robin to the CTAs.
+// Roles (384 threads): warp 0 = TMA producer, warp 1 = tcgen05 issuer of the PV products and TMEM
+// owner, warp 2 = tcgen05 issuer of the score products,
+// warps 4..7 and 8..11 = two softmax groups (thread = query row) that take the key tiles of even
+// and odd index in turn and pass the running row maximum on through shared memory, then share the
+// epilogue; warp 3 idle.
+// TMEM (512 columns): three S buffers at [0,384), used by the key tiles in turn (P, bf16, is written
+// over the first 64 columns of the tile's S buffer), O at [384,384+D).
+// Tensor-core order per key tile j:  PV(j) | S(j+3): the scores of the next tiles are ready before a
+// softmax group finishes its current tile, so both groups work without waiting for the tensor
+// cores, and rings of K and V tiles keep TMA ahead of both.
 #pragma once
 #include <type_traits>
 
@@ -14,24 +21,25 @@
 
 namespace segattn {
 
-constexpr int kFwdThreads = 192;
+constexpr int kFwdThreads = 384;
+constexpr int kFwdEwWarp0 = 4;   // first softmax warp
+constexpr int kFwdEwWarps = 8;
 constexpr float kRescaleThreshold = 8.0f;  // lazy O rescale: only when the row max grows by > 2^8
 
 template <int D>
 struct FwdSmem {
     static constexpr int kPanels = D / 64;               // 64-column (128-byte) panels per tile
     static constexpr uint32_t kTileBytes = kTile * D * 2;  // one 128-row tile of Q, K or V
+    static constexpr int kQStages = 1, kKStages = 3, kVStages = 2;
     static constexpr uint32_t kQ = 0;
-    static constexpr uint32_t kK = kTileBytes;
-    static constexpr uint32_t kV = 2 * kTileBytes;
-    static constexpr uint32_t kTotal = 3 * kTileBytes;
+    static constexpr uint32_t kK = kQStages * kTileBytes;
+    static constexpr uint32_t kV = kK + kKStages * kTileBytes;
+    static constexpr uint32_t kTotal = kV + kVStages * kTileBytes;
     static constexpr uint32_t kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
 };
 
-enum FwdBar { kBarQ = 0, kBarKFull, kBarKEmpty, kBarVFull, kBarVEmpty, kBarSFull, kBarPFull, kBarOFull, kFwdBars };
-
-// Decode blockIdx.x into a work item, heaviest first: flagged heads (long visible ranges)
-// before the others, late query tiles before early ones.
+// Decode a position in the work list into a work item, heaviest first: flagged heads (long
+// visible ranges) before the others, late query tiles before early ones.
 struct FwdItem {
     int b, hq, slot, qt;
     bool flagged;
@@ -63,40 +71,50 @@ __device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) {
     it.flagged = ht.flag[it.slot] != 0;
     return it;
 }
+// first visible key tile and number of visible key tiles of a work item
+__device__ __forceinline__ void fwd_item_tiles(const FwdParams& prm, const FwdItem& it, int* t_lo, int* n_tiles) {
+    long long jl_lo, jl_hi;
+    q_tile_kv_range(prm.geom, it.qt * kTile, it.flagged, false, &jl_lo, &jl_hi);
+    *t_lo = (int)(jl_lo / kTile);
+    *n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - *t_lo + 1 : 0;
+}
+
+// Hand-over of the running row maximum from the softmax group that finished the maximum pass of
+// tile j to the group that works on tile j + 1: named barrier 2 + (j & 1), 128 threads arrive
+// (without waiting) and 128 wait.
+__device__ __forceinline__ void fwd_m_arrive(int parity) { asm volatile("bar.arrive %0, 256;" ::"r"(2 + parity) : "memory"); }
+__device__ __forceinline__ void fwd_m_sync(int parity) { asm volatile("bar.sync %0, 256;" ::"r"(2 + parity) : "memory"); }
+// barrier of all eight softmax warps
+__device__ __forceinline__ void fwd_groups_sync() { asm volatile("bar.sync 4, 256;" ::: "memory"); }
 
 template <int D>
-__global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __grid_constant__ FwdParams prm) {
+__global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __grid_constant__ FwdParams prm) {
     using SM = FwdSmem<D>;
     constexpr int trace_id = 0;
     (void)trace_id;
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[kFwdBars];
+    constexpr int NQ = SM::kQStages, NK = SM::kKStages, NV = SM::kVStages;
+    enum { kBarQFull = 0, kBarQEmpty = kBarQFull + NQ, kBarKFull = kBarQEmpty + NQ, kBarKEmpty = kBarKFull + NK,
+           kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV, kBarSFull = kBarVEmpty + NV, kBarPFull = kBarSFull + 3,
+           kBarPvDone = kBarPFull + 2, kBarSFree = kBarPvDone + 2, kBarOFull = kBarSFree + 3, kNumBars };
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[kNumBars];
     __shared__ uint32_t tmem_slot;
+    __shared__ float s_m[2][kTile];       // [tile parity][row]: running row maximum after that tile
+    __shared__ float s_fin[2][3][kTile];  // [group][m, l, c][row]: the groups' partial sums, once per work item
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = smem_base + SM::kQ, sK = smem_base + SM::kK, sV = smem_base + SM::kV;
+    auto sQ = [&](int s) { return smem_base + SM::kQ + s * SM::kTileBytes; };
+    auto sK = [&](int s) { return smem_base + SM::kK + s * SM::kTileBytes; };
+    auto sV = [&](int s) { return smem_base + SM::kV + s * SM::kTileBytes; };
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
-
-    const FwdItem it = fwd_decode(prm, blockIdx.x);
     const MaskGeom& geo = prm.geom;
-    const int r0 = it.qt * kTile;
-    long long jl_lo, jl_hi;
-    q_tile_kv_range(geo, r0, it.flagged, false, &jl_lo, &jl_hi);
-    const int t_lo = (int)(jl_lo / kTile);
-    const int n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - t_lo + 1 : 0;
 
     if (tid == 0) {
-        mbar_init(bar(kBarQ), 1);
-        mbar_init(bar(kBarKFull), 1);
-        mbar_init(bar(kBarKEmpty), 1);
-        mbar_init(bar(kBarVFull), 1);
-        mbar_init(bar(kBarVEmpty), 1);
-        mbar_init(bar(kBarSFull), 1);
-        mbar_init(bar(kBarPFull), 128);
-        mbar_init(bar(kBarOFull), 1);
+        for (int i = 0; i < kNumBars; ++i)
+            mbar_init(bar(i), (i == kBarPFull || i == kBarPFull + 1) ? kFwdEwWarps / 2 : 1);
         fence_mbar_init();
         prefetch_tmap(&prm.tq);
         prefetch_tmap(&prm.tk);
@@ -104,241 +122,375 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
     }
     __syncwarp();
     if (warp == 1) {
-        tmem_alloc(smem_u32(&tmem_slot), 256);
+        tmem_alloc(smem_u32(&tmem_slot), 512);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
+    const uint32_t tS0 = tmem, tO = tmem + 384;
+    auto tS = [&](long long gj) { return tS0 + (uint32_t)(gj % 3) * 128; };  // S buffer of global key tile gj
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0 && n_tiles > 0) {
-            mbar_expect_tx(bar(kBarQ), SM::kTileBytes);
-            for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                tma_load_4d(sQ + pnl * 16384, &prm.tq, bar(kBarQ), pnl * 64, it.hq, r0, it.b);
-            for (int j = 0; j < n_tiles; ++j) {
-                const int row = (t_lo + j) * kTile;
-                if (!mbar_wait(bar(kBarKEmpty), (j & 1) ^ 1, 1)) break;
-                mbar_expect_tx(bar(kBarKFull), SM::kTileBytes);
-                for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                    tma_load_4d(sK + pnl * 16384, &prm.tk, bar(kBarKFull), pnl * 64, it.slot, row, it.b);
-                if (!mbar_wait(bar(kBarVEmpty), (j & 1) ^ 1, 2)) break;
-                mbar_expect_tx(bar(kBarVFull), SM::kTileBytes);
-                for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                    tma_load_4d(sV + pnl * 16384, &prm.tv, bar(kBarVFull), pnl * 64, it.slot, row, it.b);
+        if (lane == 0) {
+            int qi = blockIdx.x;  // next work item whose Q tile has not been requested yet
+            int qn_ld = 0;        // Q tiles requested so far
+            bool ok = true;
+            // request the Q tile of the next work item that has visible key tiles, if there is one
+            auto advance_q = [&]() {
+                while (ok && qi < prm.n_items) {
+                    const FwdItem it = fwd_decode(prm, qi);
+                    int t_lo, n;
+                    fwd_item_tiles(prm, it, &t_lo, &n);
+                    qi += gridDim.x;
+                    if (n == 0) continue;
+                    const int qs = qn_ld % NQ;
+                    if (!(ok = mbar_wait(bar(kBarQEmpty + qs), ((qn_ld / NQ) & 1) ^ 1, 1))) return;
+                    mbar_expect_tx(bar(kBarQFull + qs), SM::kTileBytes);
+                    for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                        tma_load_4d(sQ(qs) + pnl * 16384, &prm.tq, bar(kBarQFull + qs), pnl * 64, it.hq, it.qt * kTile, it.b);
+                    ++qn_ld;
+                    return;
+                }
+            };
+            long long g = 0;  // key tiles requested so far (all work items)
+            advance_q();
+            for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+                const FwdItem it = fwd_decode(prm, item);
+                int t_lo, n;
+                fwd_item_tiles(prm, it, &t_lo, &n);
+                if (n == 0) continue;
+                auto load_k = [&](int j) -> bool {
+                    const long long gj = g + j;
+                    const int s = (int)(gj % NK);
+                    if (!mbar_wait(bar(kBarKEmpty + s), (uint32_t)((gj / NK) & 1) ^ 1, 2)) return false;
+                    mbar_expect_tx(bar(kBarKFull + s), SM::kTileBytes);
+                    for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                        tma_load_4d(sK(s) + pnl * 16384, &prm.tk, bar(kBarKFull + s), pnl * 64, it.slot, (t_lo + j) * kTile,
+                                    it.b);
+                    return true;
+                };
+                auto load_v = [&](int j) -> bool {
+                    const long long gj = g + j;
+                    const int s = (int)(gj % NV);
+                    if (!mbar_wait(bar(kBarVEmpty + s), (uint32_t)((gj / NV) & 1) ^ 1, 3)) return false;
+                    mbar_expect_tx(bar(kBarVFull + s), SM::kTileBytes);
+                    for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                        tma_load_4d(sV(s) + pnl * 16384, &prm.tv, bar(kBarVFull + s), pnl * 64, it.slot, (t_lo + j) * kTile,
+                                    it.b);
+                    return true;
+                };
+                // K runs three tiles ahead of V, as the scores do of the PV products
+                ok = ok && load_k(0);
+                if (ok && n > 1) ok = load_k(1);
+                if (ok && n > 2) ok = load_k(2);
+                for (int j = 0; ok && j < n; ++j) {
+                    ok = load_v(j);
+                    if (ok && j + 3 < n) ok = load_k(j + 3);
+                }
+                g += n;
+                advance_q();  // the next item's Q: its buffer is free once this item's last scores are issued
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer (whole warp, uniform control flow; one elected lane issues) ----------------
-        if (n_tiles > 0) {
-            constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
-            constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
-            auto issue_qk = [&]() {
-#pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-                    mma_ss(tS, make_sdesc(sQ + off, 16, 1024), make_sdesc(sK + off, 16, 1024), idesc_qk, k > 0);
-                }
-            };
-            bool ok = warp_wait(bar(kBarQ), 0, 3) && warp_wait(bar(kBarKFull), 0, 4);
-            if (ok) {
-                tc_fence_after();
-                issue_qk();
-                mma_commit(bar(kBarKEmpty));
-                mma_commit(bar(kBarSFull));
-            }
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                ok = warp_wait(bar(kBarPFull), j & 1, 5) && warp_wait(bar(kBarVFull), j & 1, 6);
+        // ---------------- MMA issuer for O += P V (whole warp, uniform control flow; one elected lane issues) -------
+        // The two kinds of product are issued by two warps on different schedulers, so that neither
+        // waits behind the other's barriers and each has half the issue work.
+        constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
+        long long g = 0;  // key tiles of earlier work items
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+            const FwdItem it = fwd_decode(prm, item);
+            int t_lo, n;
+            fwd_item_tiles(prm, it, &t_lo, &n);
+            if (n == 0) continue;
+            for (int j = 0; ok && j < n; ++j) {
+                const long long gj = g + j;
+                const int sv = (int)(gj % NV);
+                ok = warp_wait(bar(kBarVFull + sv), (uint32_t)((gj / NV) & 1), 6) &&
+                     warp_wait(bar(kBarPFull + (int)(gj & 1)), (uint32_t)((gj >> 1) & 1), 7);
                 if (!ok) break;
                 tc_fence_after();
                 TRACE(lane == 0, j * 8 + 4);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tO, tP + k * 8, make_sdesc(sV + k * 2048, 16384, 1024), idesc_pv, (j > 0) || (k > 0));
-                mma_commit(bar(kBarVEmpty));
+                    mma_ts(tO, tS(gj) + k * 8, make_sdesc(sV(sv) + k * 2048, 16384, 1024), idesc_pv, (j > 0) || (k > 0));
+                mma_commit(bar(kBarVEmpty + sv));
+                mma_commit(bar(kBarPvDone + (int)(gj & 1)));
+                mma_commit(bar(kBarSFree + (int)(gj % 3)));  // P(j) is consumed: the S buffer may take new scores
                 TRACE(lane == 0, j * 8 + 5);
-                if (j + 1 < n_tiles) {
-                    ok = warp_wait(bar(kBarKFull), (j + 1) & 1, 7);
+            }
+            if (ok) mma_commit(bar(kBarOFull));  // the item's O is complete
+            g += n;
+        }
+    } else if (warp == 2) {
+        // ---------------- MMA issuer for S = Q K^T (whole warp; one elected lane issues) ----------------
+        constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
+        int qn = 0;       // work items with visible tiles started so far
+        long long g = 0;  // key tiles of earlier work items
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+            const FwdItem it = fwd_decode(prm, item);
+            int t_lo, n;
+            fwd_item_tiles(prm, it, &t_lo, &n);
+            if (n == 0) continue;
+            const int qs = qn % NQ;
+            if (!(ok = warp_wait(bar(kBarQFull + qs), (qn / NQ) & 1, 4))) break;
+            ++qn;
+            for (int j = 0; ok && j < n; ++j) {
+                const long long gj = g + j;
+                // the S buffer of tile gj held P of tile gj - 3: wait until that PV product has finished
+                if (gj >= 3) {
+                    ok = warp_wait(bar(kBarSFree + (int)(gj % 3)), (uint32_t)(((gj - 3) / 3) & 1), 12);
                     if (!ok) break;
                     tc_fence_after();
-                    TRACE(lane == 0, j * 8 + 6);
-                    issue_qk();
-                    TRACE(lane == 0, j * 8 + 7);
-                    mma_commit(bar(kBarKEmpty));
-                    mma_commit(bar(kBarSFull));
-                } else {
-                    mma_commit(bar(kBarOFull));
                 }
+                const int s = (int)(gj % NK);
+                if (!(ok = warp_wait(bar(kBarKFull + s), (uint32_t)((gj / NK) & 1), 5))) break;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
+                    mma_ss(tS(gj), make_sdesc(sQ(qs) + off, 16, 1024), make_sdesc(sK(s) + off, 16, 1024), idesc_qk, k > 0);
+                }
+                mma_commit(bar(kBarKEmpty + s));
+                mma_commit(bar(kBarSFull + (int)(gj % 3)));
+                if (j == n - 1) mma_commit(bar(kBarQEmpty + qs));  // the item's last scores release Q
+                TRACE(lane == 0, j * 8 + 6);
             }
+            g += n;
         }
-    } else {
-        // ---------------- softmax + epilogue: one thread per query row ----------------
-        const int row = 32 * (warp & 3) + lane;
-        const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
-        const int r = r0 + row;
-        const long long p = (long long)geo.q_pos0 + r;
-        // visible local key rows of this query row: [vlo, vhi]
-        long long vlo_ll = lo_visible(geo, p, it.flagged) - geo.kv_pos0;
-        long long vhi_ll = p - geo.kv_pos0;
-        if (vlo_ll < 0) vlo_ll = 0;
-        if (vhi_ll > geo.kv_len - 1) vhi_ll = geo.kv_len - 1;
-        const int vlo = (int)vlo_ll, vhi = (int)vhi_ll;
-        // a key tile [c0, c0+128) needs no element mask when every row of the tile sees all of it
-        long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.flagged) - geo.kv_pos0;
-        long long full_hi = (long long)geo.q_pos0 + r0 - geo.kv_pos0;
-        if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
-
+    } else if (warp >= kFwdEwWarp0) {
+        // ---------------- softmax + epilogue ----------------
+        // Two groups of four warps; thread = query row (all 128 key columns of a tile).  Group 0 takes the
+        // key tiles of even global index, group 1 the odd ones, so that one group's maximum pass and
+        // hand-offs run under the other group's exponentials.  The running maximum travels from tile to
+        // tile through shared memory; each group keeps its own partial row sum.
+        const int quarter = warp & 3, grp = (warp - kFwdEwWarp0) >> 2;
+        const int row = 32 * quarter + lane;
+        const uint32_t lane_off = (uint32_t)(32 * quarter) << 16;
+        constexpr int DH = D / 2;  // this group's share of an O row in the epilogue
         const float sl2 = prm.scale_log2;
         const uint64_t sl2x2 = f32x2(sl2, sl2);
-        // l_run: row sum of the unrounded p (gives LSE).  c_run: sum over tiles of (bf16(p) - p) for the
-        // tile's largest p.  O is divided by l_run + c_run, i.e. by a row sum in which the dominant
-        // probability enters as the bf16 value the PV product really used, so that a row where one key
-        // dominates (outlier keys) stays a convex combination of value rows.
-        float m_run = -INFINITY, l_run = 0.f, c_run = 0.f;
+        long long g = 0;  // key tiles of earlier work items
+        int qn = 0;       // earlier work items that had visible tiles
         bool ok = true;
-        // One key tile of the online softmax.  MASKED is a compile-time flag so that the common,
-        // fully visible tile runs straight-line code (no per-element tests, no branches that would keep
-        // the scheduler from overlapping the exp latency of neighbouring elements).
-        auto softmax_tile = [&](auto masked_c, const int j, const int c0) {
-            constexpr bool MASKED = decltype(masked_c)::value;
-            uint32_t va[32], vb[32];
-            // pass 1: row maximum of the raw scores; the load of chunk c+1 is in flight while chunk c is reduced
-            float mx0 = -INFINITY, mx1 = -INFINITY;
-            tmem_ld_x32(tS + lane_off, va);
+        for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+            const FwdItem it = fwd_decode(prm, item);
+            int t_lo, n_tiles;
+            fwd_item_tiles(prm, it, &t_lo, &n_tiles);
+            const int r0 = it.qt * kTile;
+            const int r = r0 + row;
+            const long long p = (long long)geo.q_pos0 + r;
+            // visible local key rows of this query row: [vlo, vhi]
+            long long vlo_ll = lo_visible(geo, p, it.flagged) - geo.kv_pos0;
+            long long vhi_ll = p - geo.kv_pos0;
+            if (vlo_ll < 0) vlo_ll = 0;
+            if (vhi_ll > geo.kv_len - 1) vhi_ll = geo.kv_len - 1;
+            const int vlo = (int)vlo_ll, vhi = (int)vhi_ll;
+            // a key tile [c0, c0+128) needs no element mask when every row of the tile sees all of it
+            long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.flagged) - geo.kv_pos0;
+            long long full_hi = (long long)geo.q_pos0 + r0 - geo.kv_pos0;
+            if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
+
+            // m_used: the running maximum this group's sums are scaled by.  l_run: sum of the unrounded p of
+            // this group's tiles (gives LSE).  c_run: sum over those tiles of (bf16(p) - p) for the tile's
+            // largest p.  O is divided by l + c, i.e. by a row sum in which the dominant probability
+            // enters as the bf16 value the PV product really used, so that a row where one key dominates
+            // (outlier keys) stays a convex combination of value rows.
+            float m_used = -INFINITY, l_run = 0.f, c_run = 0.f;
+            // One key tile of the online softmax.  MASKED is a compile-time flag so that the common,
+            // fully visible tile runs straight-line code.
+            auto softmax_tile = [&](auto masked_c, const int j, const long long gj, const int c0) {
+                constexpr bool MASKED = decltype(masked_c)::value;
+                const uint32_t tSj = tS(gj);
+                uint32_t va[32], vb[32];
+                // pass 1: row maximum of the raw scores; the load of chunk c+1 is in flight while chunk c is reduced
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+                tmem_ld_x32(tSj + lane_off, va);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t(&cur)[32] = (c & 1) ? vb : va;
-                uint32_t(&nxt)[32] = (c & 1) ? va : vb;
-                tmem_wait_ld_dep(cur);
-                tmem_ld_x32(tS + lane_off + ((c + 1) & 3) * 32, nxt);  // c == 3: chunk 0 again, for pass 2
-                if (MASKED) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int col = c0 + c * 32 + i;
-                        cur[i] = (col >= vlo && col <= vhi) ? cur[i] : 0xff800000u;  // -inf
-                    }
-                }
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    mx0 = fmax3(mx0, __uint_as_float(cur[i]), __uint_as_float(cur[i + 1]));
-                    mx1 = fmax3(mx1, __uint_as_float(cur[i + 2]), __uint_as_float(cur[i + 3]));
-                }
-            }
-            const float mx = fmaxf(mx0, mx1);
-            TRACE(tid == 64, j * 8 + 1);
-            const float m_tile = mx * sl2;  // scale > 0, so the maximum commutes with the scaling
-            const float m_new = fmaxf(m_run, m_tile);
-            const bool grow = m_new > m_run + kRescaleThreshold || (m_run == -INFINITY && m_new > -INFINITY);
-            float alpha = 1.f;
-            if (grow) {
-                alpha = ex2(m_run - m_new);  // 0 when nothing was accumulated yet
-                l_run *= alpha;
-                c_run *= alpha;
-                m_run = m_new;
-            }
-            if (j > 0 && __any_sync(0xffffffffu, grow)) {
-                // every MMA issued before this tile's S (the previous PV included) has retired
-                tmem_wait_ld_dep(va);  // the prefetched chunk 0: drain before reusing the load path
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld_x32(tO + lane_off + c * 32, v);
-                    tmem_wait_ld_dep(v);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                    tmem_st_x32(tO + lane_off + c * 32, v);
-                }
-            }
-            // pass 2: p = 2^(s*scale*log2e - m); row sum from the unrounded p; P to TMEM as bf16
-            const float m_eff = (m_run == -INFINITY) ? 0.f : m_run;
-            const uint64_t nm2 = f32x2(-m_eff, -m_eff);
-            {
-                const float pm = ex2(fmaf(mx, sl2, -m_eff));  // the tile's largest p, exactly as pass 2 forms it
-                const uint32_t pr = pack_bf16(pm, 0.f);
-                c_run += __uint_as_float(pr << 16) - pm;
-            }
-            uint64_t acc_a = 0ull, acc_b = 0ull;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t(&cur)[32] = (c & 1) ? vb : va;
-                uint32_t(&nxt)[32] = (c & 1) ? va : vb;
-                tmem_wait_ld_dep(cur);
-                if (c < 3) tmem_ld_x32(tS + lane_off + (c + 1) * 32, nxt);
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const uint64_t t = fma_f32x2(f32x2_bits(cur[i], cur[i + 1]), sl2x2, nm2);
-                    float t0, t1;
-                    f32x2_unpack(t, t0, t1);
-                    float p0 = ex2(t0), p1 = ex2(t1);
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t(&cur)[32] = (c & 1) ? vb : va;
+                    uint32_t(&nxt)[32] = (c & 1) ? va : vb;
+                    tmem_wait_ld_dep(cur);
+                    tmem_ld_x32(tSj + lane_off + ((c + 1) & 3) * 32, nxt);  // c == 3: chunk 0 again, for pass 2
                     if (MASKED) {
-                        const int col = c0 + c * 32 + i;
-                        p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
-                        p1 = (col + 1 >= vlo && col + 1 <= vhi) ? p1 : 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int col = c0 + c * 32 + i;
+                            cur[i] = (col >= vlo && col <= vhi) ? cur[i] : 0xff800000u;  // -inf
+                        }
                     }
-                    if (i & 2) acc_b = add_f32x2(acc_b, f32x2(p0, p1));
-                    else acc_a = add_f32x2(acc_a, f32x2(p0, p1));
-                    pk[i / 2] = pack_bf16(p0, p1);
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        mx0 = fmax3(mx0, __uint_as_float(cur[i]), __uint_as_float(cur[i + 1]));
+                        mx1 = fmax3(mx1, __uint_as_float(cur[i + 2]), __uint_as_float(cur[i + 3]));
+                    }
                 }
-                tmem_st_x16(tP + lane_off + c * 16, pk);
+                const float mx = fmaxf(mx0, mx1);
+                // running maximum after the previous tile (the other group's), then this tile's
+                float m_prev = -INFINITY;
+                if (j > 0) {
+                    fwd_m_sync((int)((gj - 1) & 1));
+                    m_prev = s_m[(gj - 1) & 1][row];
+                }
+                TRACE((tid & 127) == 0, j * 8 + 1);
+                const float m_tile = mx * sl2;  // scale > 0, so the maximum commutes with the scaling
+                const bool grow = m_tile > m_prev + kRescaleThreshold || (m_prev == -INFINITY && m_tile > -INFINITY);
+                const float m_new = grow ? m_tile : m_prev;
+                if (j + 1 < n_tiles) {
+                    s_m[gj & 1][row] = m_new;
+                    __threadfence_block();
+                    fwd_m_arrive((int)(gj & 1));
+                }
+                if (m_new > m_used) {  // bring this group's sums to the current scale
+                    const float f = ex2(m_used - m_new);  // 0 when nothing was accumulated yet
+                    l_run *= f;
+                    c_run *= f;
+                    m_used = m_new;
+                }
+                if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                    // PV(j-1), which accumulates into O, was issued after this tile's scores: wait for it
+                    tmem_wait_ld_dep(va);  // the prefetched chunk 0: drain before reusing the load path
+                    ok = __all_sync(0xffffffffu,
+                                    mbar_wait(bar(kBarPvDone + (int)((gj - 1) & 1)), (uint32_t)(((gj - 1) >> 1) & 1), 10));
+                    if (!ok) return;
+                    tc_fence_after();
+                    const float alpha = grow ? ex2(m_prev - m_new) : 1.f;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld_x32(tO + lane_off + c * 32, v);
+                        tmem_wait_ld_dep(v);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                        tmem_st_x32(tO + lane_off + c * 32, v);
+                    }
+                }
+                // pass 2: p = 2^(s*scale*log2e - m); row sum from the unrounded p; P to TMEM as bf16
+                const float m_eff = (m_new == -INFINITY) ? 0.f : m_new;
+                const uint64_t nm2 = f32x2(-m_eff, -m_eff);
+                {
+                    const float pm = ex2(fmaf(mx, sl2, -m_eff));  // the tile's largest p, exactly as pass 2 forms it
+                    const uint32_t pr = pack_bf16(pm, 0.f);
+                    c_run += __uint_as_float(pr << 16) - pm;
+                }
+                uint64_t acc_a = 0ull, acc_b = 0ull;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t(&cur)[32] = (c & 1) ? vb : va;
+                    uint32_t(&nxt)[32] = (c & 1) ? va : vb;
+                    tmem_wait_ld_dep(cur);
+                    if (c < 3) tmem_ld_x32(tSj + lane_off + (c + 1) * 32, nxt);
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const uint64_t t = fma_f32x2(f32x2_bits(cur[i], cur[i + 1]), sl2x2, nm2);
+                        float t0, t1;
+                        f32x2_unpack(t, t0, t1);
+                        float p0 = ex2(t0), p1 = ex2(t1);
+                        if (MASKED) {
+                            const int col = c0 + c * 32 + i;
+                            p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
+                            p1 = (col + 1 >= vlo && col + 1 <= vhi) ? p1 : 0.f;
+                        }
+                        if (i & 2) acc_b = add_f32x2(acc_b, f32x2(p0, p1));
+                        else acc_a = add_f32x2(acc_a, f32x2(p0, p1));
+                        pk[i / 2] = pack_bf16(p0, p1);
+                    }
+                    tmem_st_x16(tSj + lane_off + c * 16, pk);
+                }
+                {
+                    float s0, s1;
+                    f32x2_unpack(add_f32x2(acc_a, acc_b), s0, s1);
+                    l_run += s0 + s1;
+                }
+            };
+            for (int j = 0; j < n_tiles; ++j) {
+                const long long gj = g + j;
+                if ((int)(gj & 1) != grp) continue;  // the other group's tile
+                const int c0 = (t_lo + j) * kTile;
+                const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (int)(gj % 3)), (uint32_t)((gj / 3) & 1), 8));
+                if (!ok) break;
+                tc_fence_after();
+                TRACE((tid & 127) == 0, j * 8 + 0);
+                if (masked) softmax_tile(std::true_type{}, j, gj, c0);
+                else softmax_tile(std::false_type{}, j, gj, c0);
+                if (!ok) break;
+                tmem_wait_st();
+                // this group's previous P has been consumed (keeps the P barrier of this parity at most one
+                // completion ahead of the MMA warp; normally long since true)
+                if (gj >= 2) {
+                    ok = __all_sync(0xffffffffu,
+                                    mbar_wait(bar(kBarPvDone + (int)(gj & 1)), (uint32_t)(((gj - 2) >> 1) & 1), 11));
+                    if (!ok) break;
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarPFull + (int)(gj & 1)));
+                TRACE((tid & 127) == 0, j * 8 + 2);
             }
-            {
-                float s0, s1;
-                f32x2_unpack(add_f32x2(acc_a, acc_b), s0, s1);
-                l_run += s0 + s1;
-            }
-        };
-        for (int j = 0; j < n_tiles; ++j) {
-            const int c0 = (t_lo + j) * kTile;
-            const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull), j & 1, 8));
             if (!ok) break;
-            tc_fence_after();
-            TRACE(tid == 64, j * 8 + 0);
-            if (masked) softmax_tile(std::true_type{}, j, c0);
-            else softmax_tile(std::false_type{}, j, c0);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(kBarPFull));
-            TRACE(tid == 64, j * 8 + 2);
-        }
-        // ---------------- epilogue ----------------
-        if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), 0, 9));
-        tc_fence_after();
-        const bool have = n_tiles > 0 && ok && l_run > 0.f && l_run + c_run > 0.f;
-        const float inv_l = have ? 1.f / (l_run + c_run) : 0.f;
-        if (r < geo.Lq && (ok || n_tiles == 0)) {
-            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(prm.O) + it.b * prm.o_stride[0] +
-                                  (long long)r * prm.o_stride[1] + it.hq * prm.o_stride[2];
-            prm.LSE[((long long)it.b * prm.Hq + it.hq) * geo.Lq + r] =
-                have ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-            if (!have) {
-                for (int e = 0; e < D; e += 8) *reinterpret_cast<uint4*>(orow + e) = make_uint4(0, 0, 0, 0);
+            // ---------------- epilogue of the work item ----------------
+            float m_fin = -INFINITY, l_tot = 0.f, lc_tot = 0.f;
+            if (n_tiles > 0) {
+                // the groups combine their partial sums at the final scale
+                s_fin[grp][0][row] = m_used;
+                s_fin[grp][1][row] = l_run;
+                s_fin[grp][2][row] = c_run;
+                fwd_groups_sync();
+                const float m_o = s_fin[grp ^ 1][0][row], l_o = s_fin[grp ^ 1][1][row], c_o = s_fin[grp ^ 1][2][row];
+                m_fin = fmaxf(m_used, m_o);
+                const float f_me = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_fin);
+                const float f_o = (m_o == -INFINITY) ? 0.f : ex2(m_o - m_fin);
+                // same order of additions in both groups, so that they divide by the same number
+                const float l_g0 = grp == 0 ? l_run * f_me : l_o * f_o, l_g1 = grp == 0 ? l_o * f_o : l_run * f_me;
+                const float c_g0 = grp == 0 ? c_run * f_me : c_o * f_o, c_g1 = grp == 0 ? c_o * f_o : c_run * f_me;
+                l_tot = l_g0 + l_g1;
+                lc_tot = l_tot + (c_g0 + c_g1);
+                // one completion per work item: every PV product of the item has finished
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), (uint32_t)(qn & 1), 9));
+                if (!ok) break;
+                tc_fence_after();
+                ++qn;
             }
-        }
-        if (n_tiles > 0 && ok) {
+            const bool have = n_tiles > 0 && l_tot > 0.f && lc_tot > 0.f;
+            const float inv_l = have ? 1.f / lc_tot : 0.f;
             __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(prm.O) + it.b * prm.o_stride[0] +
-                                  (long long)r * prm.o_stride[1] + it.hq * prm.o_stride[2];
+                                  (long long)r * prm.o_stride[1] + it.hq * prm.o_stride[2] + grp * DH;
+            if (r < geo.Lq) {
+                if (grp == 0)
+                    prm.LSE[((long long)it.b * prm.Hq + it.hq) * geo.Lq + r] =
+                        have ? (m_fin + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
+                if (!have)
+                    for (int e = 0; e < DH; e += 8) *reinterpret_cast<uint4*>(orow + e) = make_uint4(0, 0, 0, 0);
+            }
+            if (n_tiles > 0) {
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_x32(tO + lane_off + c * 32, v);
-                tmem_wait_ld_dep(v);
-                if (r < geo.Lq && have) {
+                for (int c = 0; c < DH / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_x32(tO + lane_off + grp * DH + c * 32, v);
+                    tmem_wait_ld_dep(v);
+                    if (r < geo.Lq && have) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(v[i]) * inv_l, __uint_as_float(v[i + 1]) * inv_l);
-                        o.y = pack_bf16(__uint_as_float(v[i + 2]) * inv_l, __uint_as_float(v[i + 3]) * inv_l);
-                        o.z = pack_bf16(__uint_as_float(v[i + 4]) * inv_l, __uint_as_float(v[i + 5]) * inv_l);
-                        o.w = pack_bf16(__uint_as_float(v[i + 6]) * inv_l, __uint_as_float(v[i + 7]) * inv_l);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + i) = o;
+                        for (int i = 0; i < 32; i += 8) {
+                            uint4 o;
+                            o.x = pack_bf16(__uint_as_float(v[i]) * inv_l, __uint_as_float(v[i + 1]) * inv_l);
+                            o.y = pack_bf16(__uint_as_float(v[i + 2]) * inv_l, __uint_as_float(v[i + 3]) * inv_l);
+                            o.z = pack_bf16(__uint_as_float(v[i + 4]) * inv_l, __uint_as_float(v[i + 5]) * inv_l);
+                            o.w = pack_bf16(__uint_as_float(v[i + 6]) * inv_l, __uint_as_float(v[i + 7]) * inv_l);
+                            *reinterpret_cast<uint4*>(orow + c * 32 + i) = o;
+                        }
                     }
                 }
+                // Both groups have read O and the exchanged sums before either starts the next item: its
+                // first PV product (which overwrites O) needs a P arrival that comes after this barrier.
+                tc_fence_before();
+                fwd_groups_sync();
             }
+            g += n_tiles;
         }
     }
     // ---------------- teardown ----------------
@@ -347,7 +499,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2) seg_attn_fwd_kernel(const __gr
     __syncthreads();
     if (warp == 1) {
         __syncwarp();
-        tmem_dealloc(tmem, 256);
+        tmem_dealloc(tmem, 512);
     }
 }
 

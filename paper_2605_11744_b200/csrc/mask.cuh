@@ -84,6 +84,7 @@ struct alignas(64) FwdParams {
     MaskGeom geom;
     int B, Hq, g;
     int n_qtiles;
+    int n_items;       // work items: B * query heads served * n_qtiles
     float scale_log2;  // sm_scale * log2(e)
     HeadTable heads;
 };

@@ -57,6 +57,16 @@ segattn_status check_arch() {
     return major == 10 ? SEGATTN_OK : SEGATTN_ERR_UNSUPPORTED_ARCH;
 }
 
+// number of SMs of the current device
+segattn_status sm_count(int* n) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaDeviceGetAttribute(n, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return *n > 0 ? SEGATTN_OK : SEGATTN_ERR_CUDA;
+}
+
 bool strides_ok(const int64_t s[3], int d) {
     (void)d;
     for (int i = 0; i < 3; ++i)
@@ -167,14 +177,19 @@ segattn_status launch_fwd(const seg_attn_params* p, const HeadTable& heads, cons
     prm.n_qtiles = (p->Lq + kTile - 1) / kTile;
     prm.scale_log2 = p->sm_scale * 1.4426950408889634f;
     prm.heads = heads;
-    const long long grid = (long long)p->B * heads.n_slots * prm.g * prm.n_qtiles;
-    if (grid > 0x7fffffffLL) return SEGATTN_ERR_INVALID;
+    const long long n_items = (long long)p->B * heads.n_slots * prm.g * prm.n_qtiles;
+    if (n_items > 0x7fffffffLL) return SEGATTN_ERR_INVALID;
+    prm.n_items = (int)n_items;
+    // persistent: one CTA per SM walks the work list
+    int n_sm = 0;
+    if ((st = sm_count(&n_sm)) != SEGATTN_OK) return st;
+    const unsigned grid = (unsigned)(n_items < n_sm ? n_items : n_sm);
     if (p->d == 128) {
         if ((st = set_smem(seg_attn_fwd_kernel<128>, FwdSmem<128>::kDynamic)) != SEGATTN_OK) return st;
-        seg_attn_fwd_kernel<128><<<(unsigned)grid, kFwdThreads, FwdSmem<128>::kDynamic, stream>>>(prm);
+        seg_attn_fwd_kernel<128><<<grid, kFwdThreads, FwdSmem<128>::kDynamic, stream>>>(prm);
     } else {
         if ((st = set_smem(seg_attn_fwd_kernel<64>, FwdSmem<64>::kDynamic)) != SEGATTN_OK) return st;
-        seg_attn_fwd_kernel<64><<<(unsigned)grid, kFwdThreads, FwdSmem<64>::kDynamic, stream>>>(prm);
+        seg_attn_fwd_kernel<64><<<grid, kFwdThreads, FwdSmem<64>::kDynamic, stream>>>(prm);
     }
     return launch_check();
 }
