@@ -124,15 +124,28 @@ __device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) {
     return it;
 }
 
+// first visible key tile and number of visible key tiles of a work item of the dQ pass
+__device__ __forceinline__ void dq_item_tiles(const BwdParams& prm, const DqItem& it, int* t_lo, int* n_tiles) {
+    long long jl_lo, jl_hi;
+    q_tile_kv_range(prm.geom, it.qt * kTile, it.flagged, false, &jl_lo, &jl_hi);
+    *t_lo = (int)(jl_lo / kTile);
+    *n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - *t_lo + 1 : 0;
+}
+
+// Persistent: one CTA per SM walks the work list (one 128-row query tile of one (batch, query head)
+// per item, heaviest first, dealt round-robin); the rings of K and V tiles and all phase counters
+// run on across items, so that the next item's tiles arrive and its first products are issued
+// while the element-wise warps finish the current one.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const __grid_constant__ BwdParams prm) {
     using SM = DqSmem<D>;
     constexpr int trace_id = 1;
     (void)trace_id;
     constexpr int NK = SM::kKStages, NV = SM::kVStages;
-    enum { kBarQ = 0, kBarKFull = 1, kBarKEmpty = kBarKFull + NK, kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV,
-           kBarSFull = kBarVEmpty + NV, kBarDpFull = kBarSFull + 2, kBarDsFull, kBarDqFull, kNumBars };
-    extern __shared__ uint8_t smem_raw[];
+    enum { kBarQFull = 0, kBarQEmpty, kBarDoFull, kBarDoEmpty, kBarKFull, kBarKEmpty = kBarKFull + NK,
+           kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV, kBarSFull = kBarVEmpty + NV, kBarDpFull = kBarSFull + 2,
+           kBarDsFull, kBarDqFull, kNumBars };
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[kNumBars];
     __shared__ uint32_t tmem_slot;
 
@@ -142,14 +155,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
     auto sK = [&](int s) { return smem_base + SM::kK + s * SM::kTileBytes; };
     auto sV = [&](int s) { return smem_base + SM::kV + s * SM::kTileBytes; };
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
-
-    const DqItem it = dq_decode(prm, blockIdx.x);
     const MaskGeom& geo = prm.geom;
-    const int r0 = it.qt * kTile;
-    long long jl_lo, jl_hi;
-    q_tile_kv_range(geo, r0, it.flagged, false, &jl_lo, &jl_hi);
-    const int t_lo = (int)(jl_lo / kTile);
-    const int n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - t_lo + 1 : 0;
 
     if (tid == 0) {
         for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), i == kBarDsFull ? kEwWarps : 1);
@@ -172,46 +178,74 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0 && n_tiles > 0) {
-            mbar_expect_tx(bar(kBarQ), 2 * SM::kTileBytes);
-            for (int pnl = 0; pnl < SM::kPanels; ++pnl) {
-                tma_load_4d(sQ + pnl * 16384, &prm.tq, bar(kBarQ), pnl * 64, it.hq, r0, it.b);
-                tma_load_4d(sDO + pnl * 16384, &prm.tdo, bar(kBarQ), pnl * 64, it.hq, r0, it.b);
-            }
-            for (int j = 0; j < n_tiles; ++j) {
-                const int sk = j % NK, sv = j % NV;
-                const int row = (t_lo + j) * kTile;
-                if (!mbar_wait(bar(kBarKEmpty + sk), ((j / NK) & 1) ^ 1, 11)) break;
-                mbar_expect_tx(bar(kBarKFull + sk), SM::kTileBytes);
+        if (lane == 0) {
+            int qn = 0;       // work items with visible tiles started so far
+            long long g = 0;  // key tiles requested so far (all work items)
+            bool ok = true;
+            ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items_dq);
+        for (int item; ok && walk.next(&item);) {
+                const DqItem it = dq_decode(prm, item);
+                int t_lo, n;
+                dq_item_tiles(prm, it, &t_lo, &n);
+                if (n == 0) continue;
+                const int r0 = it.qt * kTile;
+                // Q is free once the previous item's last S is done; dO once the previous item's dQ, staged in
+                // the dO buffer, has been stored
+                if (!(ok = mbar_wait(bar(kBarQEmpty), (qn & 1) ^ 1, 11))) break;
+                mbar_expect_tx(bar(kBarQFull), SM::kTileBytes);
                 for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                    tma_load_4d(sK(sk) + pnl * 16384, &prm.tk, bar(kBarKFull + sk), pnl * 64, it.slot, row, it.b);
-                if (!mbar_wait(bar(kBarVEmpty + sv), ((j / NV) & 1) ^ 1, 12)) break;
-                mbar_expect_tx(bar(kBarVFull + sv), SM::kTileBytes);
+                    tma_load_4d(sQ + pnl * 16384, &prm.tq, bar(kBarQFull), pnl * 64, it.hq, r0, it.b);
+                if (!(ok = mbar_wait(bar(kBarDoEmpty), (qn & 1) ^ 1, 12))) break;
+                mbar_expect_tx(bar(kBarDoFull), SM::kTileBytes);
                 for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                    tma_load_4d(sV(sv) + pnl * 16384, &prm.tv, bar(kBarVFull + sv), pnl * 64, it.slot, row, it.b);
+                    tma_load_4d(sDO + pnl * 16384, &prm.tdo, bar(kBarDoFull), pnl * 64, it.hq, r0, it.b);
+                ++qn;
+                for (int j = 0; ok && j < n; ++j) {
+                    const long long gj = g + j;
+                    const int sk = (int)(gj % NK), sv = (int)(gj % NV);
+                    const int row = (t_lo + j) * kTile;
+                    if (!(ok = mbar_wait(bar(kBarKEmpty + sk), (uint32_t)((gj / NK) & 1) ^ 1, 11))) break;
+                    mbar_expect_tx(bar(kBarKFull + sk), SM::kTileBytes);
+                    for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                        tma_load_4d(sK(sk) + pnl * 16384, &prm.tk, bar(kBarKFull + sk), pnl * 64, it.slot, row, it.b);
+                    if (!(ok = mbar_wait(bar(kBarVEmpty + sv), (uint32_t)((gj / NV) & 1) ^ 1, 12))) break;
+                    mbar_expect_tx(bar(kBarVFull + sv), SM::kTileBytes);
+                    for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                        tma_load_4d(sV(sv) + pnl * 16384, &prm.tv, bar(kBarVFull + sv), pnl * 64, it.slot, row, it.b);
+                }
+                g += n;
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (whole warp, uniform control flow; one elected lane issues) ----------------
-        if (n_tiles > 0) {
-            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
-            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
-            // Waits on tiles brought by TMA need no tcgen05 fence; they are taken ahead of the wait on the
-            // element-wise warps so that the products of one key tile go out as one straight run of MMAs.
-            auto wait_k = [&](int j) { return warp_wait(bar(kBarKFull + j % NK), (j / NK) & 1, 14); };
-            auto wait_v = [&](int j) { return warp_wait(bar(kBarVFull + j % NV), (j / NV) & 1, 15); };
-            auto issue_s = [&](int j) {   // S(j) = Q K_j^T into the S buffer j & 1
-                const int sk = j % NK;
+        constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
+        constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
+        int qn = 0;
+        long long g = 0;  // key tiles of earlier work items
+        bool ok = true;
+        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items_dq);
+        for (int item; ok && walk.next(&item);) {
+            const DqItem it = dq_decode(prm, item);
+            int t_lo, n;
+            dq_item_tiles(prm, it, &t_lo, &n);
+            if (n == 0) continue;
+            // Waits on tiles brought by TMA need no tcgen05 fence.
+            auto wait_k = [&](int j) { return warp_wait(bar(kBarKFull + (int)((g + j) % NK)), (uint32_t)(((g + j) / NK) & 1), 14); };
+            auto wait_v = [&](int j) { return warp_wait(bar(kBarVFull + (int)((g + j) % NV)), (uint32_t)(((g + j) / NV) & 1), 15); };
+            auto issue_s = [&](int j) {   // S(j) = Q K_j^T into the S buffer of the tile's global parity
+                const long long gj = g + j;
+                const int sk = (int)(gj % NK);
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-                    mma_ss(tS0 + (j & 1) * 128, make_sdesc(sQ + off, 16, 1024), make_sdesc(sK(sk) + off, 16, 1024), idesc_s,
-                           k > 0);
+                    mma_ss(tS0 + (uint32_t)(gj & 1) * 128, make_sdesc(sQ + off, 16, 1024), make_sdesc(sK(sk) + off, 16, 1024),
+                           idesc_s, k > 0);
                 }
-                mma_commit(bar(kBarSFull + (j & 1)));
+                mma_commit(bar(kBarSFull + (int)(gj & 1)));
+                if (j == n - 1) mma_commit(bar(kBarQEmpty));   // the item's last scores release Q
             };
             auto issue_dp = [&](int j) {  // dP(j) = dO V_j^T
-                const int sv = j % NV;
+                const int sv = (int)((g + j) % NV);
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
@@ -220,158 +254,192 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                 mma_commit(bar(kBarVEmpty + sv));
                 mma_commit(bar(kBarDpFull));
             };
-            bool ok = warp_wait(bar(kBarQ), 0, 13) && wait_k(0) && wait_v(0);
-            if (ok) {
-                issue_s(0);
-                issue_dp(0);
-            }
-            if (ok && n_tiles > 1 && (ok = wait_k(1))) issue_s(1);
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                if (j + 1 < n_tiles) ok = wait_v(j + 1);
-                ok = ok && warp_wait(bar(kBarDsFull), j & 1, 16);   // dS(j) written, dP(j) read
+            ok = warp_wait(bar(kBarQFull), qn & 1, 13) && wait_k(0);
+            if (ok) issue_s(0);
+            ok = ok && warp_wait(bar(kBarDoFull), qn & 1, 13) && wait_v(0);
+            if (ok) issue_dp(0);
+            if (ok && n > 1 && (ok = wait_k(1))) issue_s(1);
+            for (int j = 0; ok && j < n; ++j) {
+                const long long gj = g + j;
+                if (j + 1 < n) ok = wait_v(j + 1);
+                ok = ok && warp_wait(bar(kBarDsFull), (uint32_t)(gj & 1), 16);   // dS(j) written, dP(j) read
                 if (!ok) break;
                 tc_fence_after();
                 TRACE(lane == 0, j * 16 + 4);
-                if (j + 1 < n_tiles) issue_dp(j + 1);   // first: phase B of the next tile waits for it
-                TRACE(lane == 0, j * 16 + 6);
-                const int sk = j % NK;
+                if (j + 1 < n) issue_dp(j + 1);   // first: phase B of the next tile waits for it
+                const int sk = (int)(gj % NK);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tDq, tS0 + (j & 1) * 128 + packed_a_col(k), make_sdesc(sK(sk) + k * 2048, 16384, 1024), idesc_dq,
-                           (j > 0) || (k > 0));
+                    mma_ts(tDq, tS0 + (uint32_t)(gj & 1) * 128 + packed_a_col(k), make_sdesc(sK(sk) + k * 2048, 16384, 1024),
+                           idesc_dq, (j > 0) || (k > 0));
                 mma_commit(bar(kBarKEmpty + sk));
-                TRACE(lane == 0, j * 16 + 7);
                 // K(j+2) reuses the stage dQ(j-1) released one run ago: its load gets the first two products
                 // of this run as extra time before it is waited for
-                if (j + 2 < n_tiles && (ok = wait_k(j + 2))) issue_s(j + 2);    // overwrites dS(j): after dQ(j)
+                if (j + 2 < n && (ok = wait_k(j + 2))) issue_s(j + 2);    // overwrites dS(j): after dQ(j)
                 TRACE(lane == 0, j * 16 + 5);
             }
             if (ok) mma_commit(bar(kBarDqFull));
+            ++qn;
+            g += n;
         }
     } else if (warp >= kEwWarp0) {
         // ---------------- element-wise: thread = query row, 64 of the tile's 128 key columns ----------------
         const int quarter = warp & 3, half = (warp - kEwWarp0) >> 2;
         const int row = 32 * quarter + lane;
         const uint32_t lane_off = (uint32_t)(32 * quarter) << 16;
-        const int r = r0 + row;
-        const long long p = (long long)geo.q_pos0 + r;
-        long long vlo_ll = lo_visible(geo, p, it.flagged) - geo.kv_pos0;
-        long long vhi_ll = p - geo.kv_pos0;
-        if (vlo_ll < 0) vlo_ll = 0;
-        if (vhi_ll > geo.kv_len - 1) vhi_ll = geo.kv_len - 1;
-        const int vlo = (int)vlo_ll, vhi = (int)vhi_ll;
-        long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.flagged) - geo.kv_pos0;
-        long long full_hi = (long long)geo.q_pos0 + r0 - geo.kv_pos0;
-        if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
-        const bool row_ok = r < geo.Lq;
-        const long long sidx = ((long long)it.b * prm.Hq + it.hq) * geo.Lq + r;
-        float lse2 = INFINITY, dsum = 0.f;  // +inf: an absent or keyless row gives P = 0
-        if (row_ok) {
-            const float l = prm.LSE[sidx];
-            lse2 = (l == -INFINITY) ? INFINITY : l * kLog2e;
-            dsum = prm.Dvec[sidx];
-        }
+        const uint32_t col_off = (uint32_t)half * 64;
         const float sl2 = prm.scale_log2;
         const uint64_t sl2x2 = f32x2(sl2, sl2);
-        const uint64_t nlse2 = f32x2(-lse2, -lse2);
-        const uint64_t ndsum2 = f32x2(-dsum, -dsum);
-        const uint32_t col_off = (uint32_t)half * 64;
-        float P[64];
-        // phase A: P = 2^(S*scale*log2e - LSE*log2e) for this thread's 64 columns of S buffer `tS`
-        auto phase_a = [&](auto masked_c, const uint32_t tS, const int c0) {
-            constexpr bool MASKED = decltype(masked_c)::value;
-            uint32_t sa_[32], sb_[32];
-            tmem_ld_x32(tS + lane_off + col_off, sa_);
-            tmem_ld_x32(tS + lane_off + col_off + 32, sb_);
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t(&sv)[32] = c ? sb_ : sa_;
-                tmem_wait_ld_dep(sv);
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float t0, t1;
-                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[i], sv[i + 1]), sl2x2, nlse2), t0, t1);
-                    float p0 = ex2(t0), p1 = ex2(t1);
-                    if (MASKED) {
-                        const int col = c0 + (int)col_off + c * 32 + i;
-                        p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
-                        p1 = (col + 1 >= vlo && col + 1 <= vhi) ? p1 : 0.f;
-                    }
-                    P[c * 32 + i] = p0;
-                    P[c * 32 + i + 1] = p1;
-                }
-            }
-        };
-        // phase B: dS = P * (dP - D), rounded to bf16, written over the start of this half of the tile's S
-        // buffer (its scores went into P in phase A; the next product into that buffer is issued after dQ)
-        auto phase_b = [&](const uint32_t tS) {
-            uint32_t da_[32], db_[32];
-            tmem_ld_x32(tDp + lane_off + col_off, da_);
-            tmem_ld_x32(tDp + lane_off + col_off + 32, db_);
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t(&dv)[32] = c ? db_ : da_;
-                tmem_wait_ld_dep(dv);
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const uint64_t ds2 = mul_f32x2(f32x2(P[c * 32 + i], P[c * 32 + i + 1]),
-                                                   add_f32x2(f32x2_bits(dv[i], dv[i + 1]), ndsum2));
-                    float d0, d1;
-                    f32x2_unpack(ds2, d0, d1);
-                    pk[i / 2] = pack_bf16(d0, d1);
-                }
-                tmem_st_x16(tS + lane_off + col_off + c * 16, pk);
-            }
-        };
-        bool ok = true;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int c0 = (t_lo + j) * kTile;
-            const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (j & 1)), (j >> 1) & 1, 17));
-            if (!ok) break;
-            tc_fence_after();
-            TRACE(tid == 128, j * 16 + 0);
-            if (masked) phase_a(std::true_type{}, tS0 + (j & 1) * 128, c0);
-            else phase_a(std::false_type{}, tS0 + (j & 1) * 128, c0);
-            TRACE(tid == 128, j * 16 + 1);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDpFull), j & 1, 19));
-            if (!ok) break;
-            tc_fence_after();
-            TRACE(tid == 128, j * 16 + 2);
-            phase_b(tS0 + (j & 1) * 128);
-            tmem_wait_st();
-            ew_warp_arrive(bar(kBarDsFull), lane);
-            TRACE(tid == 128, j * 16 + 3);
-            TRACE(lane == 0, j * 16 + 8 + (warp - kEwWarp0));
-        }
-        if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDqFull), 0, 18));
-        tc_fence_after();
         constexpr int DH = D / 2;  // this thread's share of the row
-        __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(prm.dQ) + it.b * prm.q_stride[0] +
-                              (long long)r * prm.q_stride[1] + it.hq * prm.q_stride[2] + half * DH;
-        if (n_tiles == 0) {
-            if (row_ok)
-                for (int e = 0; e < DH; e += 8) *reinterpret_cast<uint4*>(grow + e) = make_uint4(0, 0, 0, 0);
-        } else if (ok) {
-            const float sc = prm.sm_scale;
+        int qn = 0;
+        long long g = 0;  // key tiles of earlier work items
+        bool ok = true;
+        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items_dq);
+        for (int item; ok && walk.next(&item);) {
+            const DqItem it = dq_decode(prm, item);
+            int t_lo, n_tiles;
+            dq_item_tiles(prm, it, &t_lo, &n_tiles);
+            const int r0 = it.qt * kTile;
+            const int r = r0 + row;
+            const long long p = (long long)geo.q_pos0 + r;
+            long long vlo_ll = lo_visible(geo, p, it.flagged) - geo.kv_pos0;
+            long long vhi_ll = p - geo.kv_pos0;
+            if (vlo_ll < 0) vlo_ll = 0;
+            if (vhi_ll > geo.kv_len - 1) vhi_ll = geo.kv_len - 1;
+            const int vlo = (int)vlo_ll, vhi = (int)vhi_ll;
+            long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.flagged) - geo.kv_pos0;
+            long long full_hi = (long long)geo.q_pos0 + r0 - geo.kv_pos0;
+            if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
+            const bool row_ok = r < geo.Lq;
+            const long long sidx = ((long long)it.b * prm.Hq + it.hq) * geo.Lq + r;
+            float lse2 = INFINITY, dsum = 0.f;  // +inf: an absent or keyless row gives P = 0
+            if (row_ok) {
+                const float l = prm.LSE[sidx];
+                lse2 = (l == -INFINITY) ? INFINITY : l * kLog2e;
+                dsum = prm.Dvec[sidx];
+            }
+            const uint64_t nlse2 = f32x2(-lse2, -lse2);
+            const uint64_t ndsum2 = f32x2(-dsum, -dsum);
+            float P[64];
+            // phase A: P = 2^(S*scale*log2e - LSE*log2e) for this thread's 64 columns of S buffer `tS`
+            auto phase_a = [&](auto masked_c, const uint32_t tS, const int c0) {
+                constexpr bool MASKED = decltype(masked_c)::value;
+                uint32_t sa_[32], sb_[32];
+                tmem_ld_x32(tS + lane_off + col_off, sa_);
+                tmem_ld_x32(tS + lane_off + col_off + 32, sb_);
 #pragma unroll
-            for (int c = 0; c < DH / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_x32(tDq + lane_off + half * DH + c * 32, v);
-                tmem_wait_ld_dep(v);
-                if (row_ok) {
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t(&sv)[32] = c ? sb_ : sa_;
+                    tmem_wait_ld_dep(sv);
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float t0, t1;
+                        f32x2_unpack(fma_f32x2(f32x2_bits(sv[i], sv[i + 1]), sl2x2, nlse2), t0, t1);
+                        float p0 = ex2(t0), p1 = ex2(t1);
+                        if (MASKED) {
+                            const int col = c0 + (int)col_off + c * 32 + i;
+                            p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
+                            p1 = (col + 1 >= vlo && col + 1 <= vhi) ? p1 : 0.f;
+                        }
+                        P[c * 32 + i] = p0;
+                        P[c * 32 + i + 1] = p1;
+                    }
+                }
+            };
+            // phase B: dS = P * (dP - D), rounded to bf16, written over the start of this half of the tile's S
+            // buffer (its scores went into P in phase A; the next product into that buffer is issued after dQ)
+            auto phase_b = [&](const uint32_t tS) {
+                uint32_t da_[32], db_[32];
+                tmem_ld_x32(tDp + lane_off + col_off, da_);
+                tmem_ld_x32(tDp + lane_off + col_off + 32, db_);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t(&dv)[32] = c ? db_ : da_;
+                    tmem_wait_ld_dep(dv);
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const uint64_t ds2 = mul_f32x2(f32x2(P[c * 32 + i], P[c * 32 + i + 1]),
+                                                       add_f32x2(f32x2_bits(dv[i], dv[i + 1]), ndsum2));
+                        float d0, d1;
+                        f32x2_unpack(ds2, d0, d1);
+                        pk[i / 2] = pack_bf16(d0, d1);
+                    }
+                    tmem_st_x16(tS + lane_off + col_off + c * 16, pk);
+                }
+            };
+            for (int j = 0; j < n_tiles; ++j) {
+                const long long gj = g + j;
+                const uint32_t tS = tS0 + (uint32_t)(gj & 1) * 128;
+                const int c0 = (t_lo + j) * kTile;
+                const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (int)(gj & 1)), (uint32_t)((gj >> 1) & 1), 17));
+                if (!ok) break;
+                tc_fence_after();
+                TRACE(tid == 128, j * 16 + 0);
+                if (masked) phase_a(std::true_type{}, tS, c0);
+                else phase_a(std::false_type{}, tS, c0);
+                TRACE(tid == 128, j * 16 + 1);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDpFull), (uint32_t)(gj & 1), 19));
+                if (!ok) break;
+                tc_fence_after();
+                TRACE(tid == 128, j * 16 + 2);
+                phase_b(tS);
+                tmem_wait_st();
+                ew_warp_arrive(bar(kBarDsFull), lane);
+                TRACE(tid == 128, j * 16 + 3);
+            }
+            if (!ok) break;
+            if (n_tiles > 0) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarDqFull), (uint32_t)(qn & 1), 18));
+                if (!ok) break;
+                tc_fence_after();
+                ++qn;
+            }
+            __nv_bfloat16* grow = reinterpret_cast<__nv_bfloat16*>(prm.dQ) + it.b * prm.q_stride[0] +
+                                  (long long)r * prm.q_stride[1] + it.hq * prm.q_stride[2] + half * DH;
+            if (n_tiles == 0) {
+                if (row_ok)
+                    for (int e = 0; e < DH; e += 8) *reinterpret_cast<uint4*>(grow + e) = make_uint4(0, 0, 0, 0);
+            } else {
+                // dQ goes out through shared memory and one tiled TMA store per 64-column panel (a row-per-thread
+                // store straight to global would touch 32 different lines per instruction).  The staging tile is
+                // the dO buffer: every product that reads it has finished, and the producer may refill it only
+                // after the arrival below.
+                const float sc = prm.sm_scale;
+                constexpr int kChunks = DH / 8;                       // 16-byte chunks this thread writes
+                const int chunk0 = (half * DH % 64) / 8;              // first chunk inside the 128-byte panel row
+                const uint32_t st_row = sDO + (uint32_t)((half * DH) / 64) * 16384 + (uint32_t)row * 128;
+#pragma unroll
+                for (int c = 0; c < DH / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_x32(tDq + lane_off + half * DH + c * 32, v);
+                    tmem_wait_ld_dep(v);
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(v[i]) * sc, __uint_as_float(v[i + 1]) * sc);
-                        o.y = pack_bf16(__uint_as_float(v[i + 2]) * sc, __uint_as_float(v[i + 3]) * sc);
-                        o.z = pack_bf16(__uint_as_float(v[i + 4]) * sc, __uint_as_float(v[i + 5]) * sc);
-                        o.w = pack_bf16(__uint_as_float(v[i + 6]) * sc, __uint_as_float(v[i + 7]) * sc);
-                        *reinterpret_cast<uint4*>(grow + c * 32 + i) = o;
+                        const uint32_t x = pack_bf16(__uint_as_float(v[i]) * sc, __uint_as_float(v[i + 1]) * sc);
+                        const uint32_t y = pack_bf16(__uint_as_float(v[i + 2]) * sc, __uint_as_float(v[i + 3]) * sc);
+                        const uint32_t z = pack_bf16(__uint_as_float(v[i + 4]) * sc, __uint_as_float(v[i + 5]) * sc);
+                        const uint32_t w = pack_bf16(__uint_as_float(v[i + 6]) * sc, __uint_as_float(v[i + 7]) * sc);
+                        const int ch = chunk0 + c * 4 + i / 8;
+                        st_shared_v4(st_row + (uint32_t)((ch ^ (row & 7)) << 4), x, y, z, w);
                     }
                 }
+                (void)kChunks;
+                // the next item's first dQ product overwrites the accumulator; it is issued only after this
+                // warp's next arrival on the dS barrier, which comes after the loads above
+                tc_fence_before();
+                fence_proxy_async_smem();
+                ew_bar_sync();
+                if (tid == kEwWarp0 * 32) {
+                    for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                        tma_store_4d(&prm.tdq, sDO + pnl * 16384, pnl * 64, it.hq, r0, it.b);
+                    bulk_commit_group();
+                    bulk_wait_read_all();
+                    mbar_arrive(bar(kBarDoEmpty));   // the dO buffer may take the next item's tile
+                }
             }
+            g += n_tiles;
         }
     }
     drain_if_failed();

@@ -135,16 +135,16 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            int qi = blockIdx.x;  // next work item whose Q tile has not been requested yet
+            ItemWalk q_walk(blockIdx.x, gridDim.x, prm.n_items);  // runs ahead: the next item whose Q is not requested yet
             int qn_ld = 0;        // Q tiles requested so far
             bool ok = true;
             // request the Q tile of the next work item that has visible key tiles, if there is one
             auto advance_q = [&]() {
-                while (ok && qi < prm.n_items) {
+                int qi;
+                while (ok && q_walk.next(&qi)) {
                     const FwdItem it = fwd_decode(prm, qi);
                     int t_lo, n;
                     fwd_item_tiles(prm, it, &t_lo, &n);
-                    qi += gridDim.x;
                     if (n == 0) continue;
                     const int qs = qn_ld % NQ;
                     if (!(ok = mbar_wait(bar(kBarQEmpty + qs), ((qn_ld / NQ) & 1) ^ 1, 1))) return;
@@ -157,7 +157,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             };
             long long g = 0;  // key tiles requested so far (all work items)
             advance_q();
-            for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+            ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
+        for (int item; ok && walk.next(&item);) {
                 const FwdItem it = fwd_decode(prm, item);
                 int t_lo, n;
                 fwd_item_tiles(prm, it, &t_lo, &n);
@@ -201,7 +202,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
         long long g = 0;  // key tiles of earlier work items
         bool ok = true;
-        for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
+        for (int item; ok && walk.next(&item);) {
             const FwdItem it = fwd_decode(prm, item);
             int t_lo, n;
             fwd_item_tiles(prm, it, &t_lo, &n);
@@ -231,7 +233,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         int qn = 0;       // work items with visible tiles started so far
         long long g = 0;  // key tiles of earlier work items
         bool ok = true;
-        for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
+        for (int item; ok && walk.next(&item);) {
             const FwdItem it = fwd_decode(prm, item);
             int t_lo, n;
             fwd_item_tiles(prm, it, &t_lo, &n);
@@ -276,7 +279,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         long long g = 0;  // key tiles of earlier work items
         int qn = 0;       // earlier work items that had visible tiles
         bool ok = true;
-        for (int item = blockIdx.x; ok && item < prm.n_items; item += gridDim.x) {
+        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
+        for (int item; ok && walk.next(&item);) {
             const FwdItem it = fwd_decode(prm, item);
             int t_lo, n_tiles;
             fwd_item_tiles(prm, it, &t_lo, &n_tiles);
@@ -300,6 +304,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             // enters as the bf16 value the PV product really used, so that a row where one key dominates
             // (outlier keys) stays a convex combination of value rows.
             float m_used = -INFINITY, l_run = 0.f, c_run = 0.f;
+            TRACE(tid == 128, 2048 + qn * 4 + 0);
             // One key tile of the online softmax.  MASKED is a compile-time flag so that the common,
             // fully visible tile runs straight-line code.
             auto softmax_tile = [&](auto masked_c, const int j, const long long gj, const int c0) {
@@ -433,6 +438,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 TRACE((tid & 127) == 0, j * 8 + 2);
             }
             if (!ok) break;
+            TRACE(tid == 128, 2048 + qn * 4 + 1);
             // ---------------- epilogue of the work item ----------------
             float m_fin = -INFINITY, l_tot = 0.f, lc_tot = 0.f;
             if (n_tiles > 0) {
@@ -454,6 +460,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), (uint32_t)(qn & 1), 9));
                 if (!ok) break;
                 tc_fence_after();
+                TRACE(tid == 128, 2048 + qn * 4 + 2);
                 ++qn;
             }
             const bool have = n_tiles > 0 && l_tot > 0.f && lc_tot > 0.f;
@@ -489,6 +496,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 // first PV product (which overwrites O) needs a P arrival that comes after this barrier.
                 tc_fence_before();
                 fwd_groups_sync();
+                TRACE(tid == 128, 2048 + (qn - 1) * 4 + 3);
             }
             g += n_tiles;
         }

@@ -76,8 +76,28 @@ struct HeadTable {
     int n_slots, n_flagged;
 };
 
+// The work items a persistent CTA takes, in order: the list is sorted heaviest first and dealt to the
+// CTAs in rounds, every other round in reverse CTA order, so that no CTA always gets the heaviest item
+// of a round.
+struct ItemWalk {
+    int k, c, G, n;
+    __device__ ItemWalk(int cta, int n_ctas, int n_items) : k(0), c(cta), G(n_ctas), n(n_items) {}
+    __device__ bool next(int* item) {
+        while ((long long)k * G < n) {
+            const int i = k * G + ((k & 1) ? G - 1 - c : c);
+            ++k;
+            if (i < n) {
+                *item = i;
+                return true;
+            }
+        }
+        return false;
+    }
+};
+
 struct alignas(64) FwdParams {
     CUtensorMap tq, tk, tv;  // bf16 (d, heads, rows, batch), box (64, 1, 128, 1), 128-byte swizzle
+    CUtensorMap to;          // O, for tiled stores
     void* O;
     float* LSE;
     long long o_stride[3];
@@ -91,6 +111,7 @@ struct alignas(64) FwdParams {
 
 struct alignas(64) BwdParams {
     CUtensorMap tq, tk, tv, tdo;  // same form as above
+    CUtensorMap tdq, tdk, tdv;    // the gradient tensors, for tiled stores
     const float* LSE;             // [B][Hq][Lq]
     const float* Dvec;            // [B][Hq][Lq]  row dots <dO, O>
     void* dQ;
@@ -100,6 +121,7 @@ struct alignas(64) BwdParams {
     MaskGeom geom;
     int B, Hq, Hkv, g;
     int n_qtiles, n_kvtiles;
+    int n_items_dq;    // work items of the dQ pass: B * query heads served * n_qtiles
     float scale_log2;  // sm_scale * log2(e)
     float sm_scale;
     HeadTable heads;

@@ -167,6 +167,7 @@ segattn_status launch_fwd(const seg_attn_params* p, const HeadTable& heads, cons
     if ((st = make_map(&prm.tv, vbase, p->d, heads.n_slots, p->kv_len, p->B, p->kv_len > 0 ? p->v_stride : p->q_stride)) !=
         SEGATTN_OK)
         return st;
+    if ((st = make_map(&prm.to, O, p->d, p->Hq, p->Lq, p->B, p->o_stride)) != SEGATTN_OK) return st;
     prm.O = O;
     prm.LSE = LSE;
     for (int i = 0; i < 3; ++i) prm.o_stride[i] = p->o_stride[i];
