@@ -751,30 +751,42 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
                     *reinterpret_cast<uint4*>(gv + e) = make_uint4(0, 0, 0, 0);
                 }
         } else if (ok) {
+            // dV and dK go out through shared memory (the first dO and Q stages, idle by now) and tiled TMA
+            // stores: a row-per-thread store straight to global would touch 32 different lines per instruction.
+            // Rows past the end of the tensors are clipped by the stores.
             const float sc = prm.sm_scale;
+            const int chunk0 = (half * DH % 64) / 8;  // first 16-byte chunk inside the 128-byte panel row
+            const uint32_t row_off = (uint32_t)((half * DH) / 64) * 16384 + (uint32_t)row * 128;
 #pragma unroll
             for (int c = 0; c < DH / 32; ++c) {
                 uint32_t v[32], k[32];
                 tmem_ld_x32(tDv + lane_off + half * DH + c * 32, v);
                 tmem_ld_x32(tDk + lane_off + half * DH + c * 32, k);
                 tmem_wait_ld();
-                if (row_ok) {
 #pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
-                        o.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-                        o.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
-                        o.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
-                        *reinterpret_cast<uint4*>(gv + c * 32 + e) = o;
-                        o.x = pack_bf16(__uint_as_float(k[e]) * sc, __uint_as_float(k[e + 1]) * sc);
-                        o.y = pack_bf16(__uint_as_float(k[e + 2]) * sc, __uint_as_float(k[e + 3]) * sc);
-                        o.z = pack_bf16(__uint_as_float(k[e + 4]) * sc, __uint_as_float(k[e + 5]) * sc);
-                        o.w = pack_bf16(__uint_as_float(k[e + 6]) * sc, __uint_as_float(k[e + 7]) * sc);
-                        *reinterpret_cast<uint4*>(gk + c * 32 + e) = o;
-                    }
+                for (int e = 0; e < 32; e += 8) {
+                    const uint32_t sw = (uint32_t)(((chunk0 + c * 4 + e / 8) ^ (row & 7)) << 4);
+                    st_shared_v4(sDO(0) + row_off + sw, pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
+                                 pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
+                                 pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
+                                 pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
+                    st_shared_v4(sQ(0) + row_off + sw, pack_bf16(__uint_as_float(k[e]) * sc, __uint_as_float(k[e + 1]) * sc),
+                                 pack_bf16(__uint_as_float(k[e + 2]) * sc, __uint_as_float(k[e + 3]) * sc),
+                                 pack_bf16(__uint_as_float(k[e + 4]) * sc, __uint_as_float(k[e + 5]) * sc),
+                                 pack_bf16(__uint_as_float(k[e + 6]) * sc, __uint_as_float(k[e + 7]) * sc));
                 }
             }
+            fence_proxy_async_smem();
+        }
+        // every element-wise thread reaches this barrier (also after a failed wait or with nothing to do)
+        ew_bar_sync();
+        if (tid == kEwWarp0 * 32 && n_it > 0 && ok) {
+            for (int pnl = 0; pnl < SM::kPanels; ++pnl) {
+                tma_store_4d(&prm.tdv, sDO(0) + pnl * 16384, pnl * 64, slot, c0, b);
+                tma_store_4d(&prm.tdk, sQ(0) + pnl * 16384, pnl * 64, slot, c0, b);
+            }
+            bulk_commit_group();
+            bulk_wait_all();
         }
     }
     drain_if_failed();

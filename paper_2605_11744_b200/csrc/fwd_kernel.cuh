@@ -30,11 +30,12 @@ template <int D>
 struct FwdSmem {
     static constexpr int kPanels = D / 64;               // 64-column (128-byte) panels per tile
     static constexpr uint32_t kTileBytes = kTile * D * 2;  // one 128-row tile of Q, K or V
-    static constexpr int kQStages = 1, kKStages = 3, kVStages = 2;
+    static constexpr int kQStages = 1, kKStages = 2, kVStages = 2;
     static constexpr uint32_t kQ = 0;
     static constexpr uint32_t kK = kQStages * kTileBytes;
     static constexpr uint32_t kV = kK + kKStages * kTileBytes;
-    static constexpr uint32_t kTotal = kV + kVStages * kTileBytes;
+    static constexpr uint32_t kOut = kV + kVStages * kTileBytes;  // staging tile of O for the tiled store
+    static constexpr uint32_t kTotal = kOut + kTileBytes;
     static constexpr uint32_t kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
 };
 
@@ -109,10 +110,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     auto sQ = [&](int s) { return smem_base + SM::kQ + s * SM::kTileBytes; };
     auto sK = [&](int s) { return smem_base + SM::kK + s * SM::kTileBytes; };
     auto sV = [&](int s) { return smem_base + SM::kV + s * SM::kTileBytes; };
+    const uint32_t sOut = smem_base + SM::kOut;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     const MaskGeom& geo = prm.geom;
 
     if (tid == 0) {
+        prefetch_tmap(&prm.to);
         for (int i = 0; i < kNumBars; ++i)
             mbar_init(bar(i), (i == kBarPFull || i == kBarPFull + 1) ? kFwdEwWarps / 2 : 1);
         fence_mbar_init();
@@ -442,6 +445,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             // ---------------- epilogue of the work item ----------------
             float m_fin = -INFINITY, l_tot = 0.f, lc_tot = 0.f;
             if (n_tiles > 0) {
+                // the previous item's O tile has left the staging buffer
+                if (tid == kFwdEwWarp0 * 32) bulk_wait_read_all();
                 // the groups combine their partial sums at the final scale
                 s_fin[grp][0][row] = m_used;
                 s_fin[grp][1][row] = l_run;
@@ -465,43 +470,52 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             }
             const bool have = n_tiles > 0 && l_tot > 0.f && lc_tot > 0.f;
             const float inv_l = have ? 1.f / lc_tot : 0.f;
-            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(prm.O) + it.b * prm.o_stride[0] +
-                                  (long long)r * prm.o_stride[1] + it.hq * prm.o_stride[2] + grp * DH;
-            if (r < geo.Lq) {
-                if (grp == 0)
-                    prm.LSE[((long long)it.b * prm.Hq + it.hq) * geo.Lq + r] =
-                        have ? (m_fin + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
-                if (!have)
+            if (r < geo.Lq && grp == 0)
+                prm.LSE[((long long)it.b * prm.Hq + it.hq) * geo.Lq + r] =
+                    have ? (m_fin + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
+            if (n_tiles == 0) {
+                __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(prm.O) + it.b * prm.o_stride[0] +
+                                      (long long)r * prm.o_stride[1] + it.hq * prm.o_stride[2] + grp * DH;
+                if (r < geo.Lq)
                     for (int e = 0; e < DH; e += 8) *reinterpret_cast<uint4*>(orow + e) = make_uint4(0, 0, 0, 0);
-            }
-            if (n_tiles > 0) {
+            } else {
+                // O goes out through shared memory and one tiled TMA store per 64-column panel (a row-per-thread
+                // store straight to global would touch 32 different lines per instruction); rows past the end
+                // of the tensor are clipped by the store
+                const int chunk0 = (grp * DH % 64) / 8;  // first 16-byte chunk inside the 128-byte panel row
+                const uint32_t st_row = sOut + (uint32_t)((grp * DH) / 64) * 16384 + (uint32_t)row * 128;
 #pragma unroll
                 for (int c = 0; c < DH / 32; ++c) {
                     uint32_t v[32];
                     tmem_ld_x32(tO + lane_off + grp * DH + c * 32, v);
                     tmem_wait_ld_dep(v);
-                    if (r < geo.Lq && have) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 8) {
-                            uint4 o;
-                            o.x = pack_bf16(__uint_as_float(v[i]) * inv_l, __uint_as_float(v[i + 1]) * inv_l);
-                            o.y = pack_bf16(__uint_as_float(v[i + 2]) * inv_l, __uint_as_float(v[i + 3]) * inv_l);
-                            o.z = pack_bf16(__uint_as_float(v[i + 4]) * inv_l, __uint_as_float(v[i + 5]) * inv_l);
-                            o.w = pack_bf16(__uint_as_float(v[i + 6]) * inv_l, __uint_as_float(v[i + 7]) * inv_l);
-                            *reinterpret_cast<uint4*>(orow + c * 32 + i) = o;
-                        }
+                    for (int i = 0; i < 32; i += 8) {
+                        const uint32_t x = pack_bf16(__uint_as_float(v[i]) * inv_l, __uint_as_float(v[i + 1]) * inv_l);
+                        const uint32_t y = pack_bf16(__uint_as_float(v[i + 2]) * inv_l, __uint_as_float(v[i + 3]) * inv_l);
+                        const uint32_t z = pack_bf16(__uint_as_float(v[i + 4]) * inv_l, __uint_as_float(v[i + 5]) * inv_l);
+                        const uint32_t w = pack_bf16(__uint_as_float(v[i + 6]) * inv_l, __uint_as_float(v[i + 7]) * inv_l);
+                        const int ch = chunk0 + c * 4 + i / 8;
+                        st_shared_v4(st_row + (uint32_t)((ch ^ (row & 7)) << 4), x, y, z, w);
                     }
                 }
                 // Both groups have read O and the exchanged sums before either starts the next item: its
                 // first PV product (which overwrites O) needs a P arrival that comes after this barrier.
                 tc_fence_before();
+                fence_proxy_async_smem();
                 fwd_groups_sync();
+                if (tid == kFwdEwWarp0 * 32) {
+                    for (int pnl = 0; pnl < SM::kPanels; ++pnl)
+                        tma_store_4d(&prm.to, sOut + pnl * 16384, pnl * 64, it.hq, r0, it.b);
+                    bulk_commit_group();
+                }
                 TRACE(tid == 128, 2048 + (qn - 1) * 4 + 3);
             }
             g += n_tiles;
         }
     }
     // ---------------- teardown ----------------
+    if (tid == kFwdEwWarp0 * 32) bulk_wait_all();  // the last O tile has been written
     drain_if_failed();
     tc_fence_before();
     __syncthreads();

@@ -24,8 +24,13 @@ struct MaskGeom {
     int Lq, kv_len;
 };
 
+// p / S for a non-negative position: positions fit 32 bits in practice, and a 32-bit division is
+// several times cheaper on the device than a 64-bit one (these run per work item in every thread)
+__host__ __device__ inline long long seg_of(long long p, int S) {
+    return p <= 0xffffffffLL ? (long long)((unsigned)p / (unsigned)S) : p / S;
+}
 __host__ __device__ inline long long tail_start(const MaskGeom& g, long long p) {
-    long long a = (p / g.S) * (long long)g.S - g.T;
+    long long a = seg_of(p, g.S) * (long long)g.S - g.T;
     return a < 0 ? 0 : a;
 }
 __host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, bool flagged) {
@@ -33,7 +38,7 @@ __host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, 
 }
 // one past the last query position that differentiably reads key position j
 __host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j) {
-    long long seg_end = (j / g.S + 1) * (long long)g.S;
+    long long seg_end = (seg_of(j, g.S) + 1) * (long long)g.S;
     return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
 }
 
