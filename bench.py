@@ -37,9 +37,9 @@ UNIT = "TFLOP/s"
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on the
 # benchmark workload, taken from the ncu captures summarised under profiles/; None = not captured.
 NCU_TRAFFIC_BYTES = {
-    ("cfg2_gqa16k", "fwd"): None,
-    ("cfg2_gqa16k", "dq"): None,
-    ("cfg2_gqa16k", "dkv"): None,
+    ("cfg2_gqa16k", "fwd"): 651273216,
+    ("cfg2_gqa16k", "dq"): 938126848,
+    ("cfg2_gqa16k", "dkv"): 804103424,
 }
 
 
@@ -369,7 +369,7 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="benchmark configuration number (1-5); default 2")
