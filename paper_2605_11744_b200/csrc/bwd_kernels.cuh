@@ -496,10 +496,21 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
     auto sDO = [&](int s) { return smem_base + SM::kDO + s * SM::kTileBytes; };
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
-    // work item: key tiles in reverse order (late tiles first), then KV head, then batch
-    const int kt = prm.n_kvtiles - 1 - (int)(blockIdx.x % prm.n_kvtiles);
-    const int slot = (int)((blockIdx.x / prm.n_kvtiles) % prm.heads.n_slots);
-    const int b = (int)(blockIdx.x / ((long long)prm.n_kvtiles * prm.heads.n_slots));
+    // Work item: the grid is laid out as (KV head, batch) x (segment) x (rank of the tile inside its
+    // segment).  Neighbouring CTAs thus read the same query tiles (L2 reuse), and inside a segment the
+    // heavy tiles come first: the tiles of the carried tail (read by two segments), then the segment's
+    // tiles from its first on (the earlier the tile, the more query tiles follow it), so that the grid
+    // ends with short items.  Positions past the last key tile are empty.
+    const int n_bs = prm.heads.n_slots * prm.B;
+    const int rank = (int)(blockIdx.x % (unsigned)prm.dkv_tps);
+    const int rem = (int)(blockIdx.x / (unsigned)prm.dkv_tps);
+    const int seg = rem % prm.dkv_n_seg, bs = rem / prm.dkv_n_seg;
+    (void)n_bs;
+    const int k_in_seg = rank < prm.dkv_tail_tiles ? prm.dkv_tps - prm.dkv_tail_tiles + rank : rank - prm.dkv_tail_tiles;
+    const int kt = seg * prm.dkv_tps + k_in_seg;
+    if (kt >= prm.n_kvtiles) return;
+    const int slot = bs % prm.heads.n_slots;
+    const int b = bs / prm.heads.n_slots;
     const int hq0 = prm.heads.logical[slot] * prm.g;
     const MaskGeom& geo = prm.geom;
     const int c0 = kt * kTile;

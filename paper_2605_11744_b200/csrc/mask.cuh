@@ -127,6 +127,7 @@ struct alignas(64) BwdParams {
     int B, Hq, Hkv, g;
     int n_qtiles, n_kvtiles;
     int n_items_dq;    // work items of the dQ pass: B * query heads served * n_qtiles
+    int dkv_tps, dkv_tail_tiles, dkv_n_seg;  // dK/dV grid: key tiles per segment, of which in the tail, segments
     float scale_log2;  // sm_scale * log2(e)
     float sm_scale;
     HeadTable heads;
