@@ -56,6 +56,13 @@ typedef enum {
     SEGATTN_ERR_TOO_LARGE = 6         /* problem exceeds the fixed scratch of seg_attn_bwd_static */
 } segattn_status;
 
+/* seg_attn_params.flags, bit 0: for flagged KV heads the reads of the carried tail are stop-gradient
+ * too, i.e. diff(p, j) <=> i*S <= j <= p for them.  This is the literal reading of Appendix C,
+ * Eq. "ctx", where only local heads build and read the differentiable carried state and long-range
+ * heads see their prefix forward-only.  The forward is the same in both readings; only the set of
+ * (query, key) pairs that feed dK/dV changes. */
+#define SEGATTN_FLAG_FLAGGED_TAIL_SG 1
+
 typedef struct {
     int32_t B;       /* batch */
     int32_t Lq;      /* number of query rows per batch element */
@@ -68,7 +75,7 @@ typedef struct {
     int32_t q_pos0;  /* global position of query row 0 (0 for a whole sequence; i*S when streaming) */
     int32_t kv_pos0; /* global position of key row 0 (may be negative: rows before position 0 are never visible) */
     float sm_scale;  /* softmax scale; the paper uses 1/sqrt(d) */
-    int32_t reserved;
+    int32_t flags;   /* bit set of SEGATTN_FLAG_*; 0 for the default semantics */
     int64_t q_stride[3]; /* element strides of Q (and dQ) for (batch, position, head) */
     int64_t k_stride[3]; /* element strides of K (and dK) */
     int64_t v_stride[3]; /* element strides of V (and dV) */

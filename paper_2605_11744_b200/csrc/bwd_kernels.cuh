@@ -515,7 +515,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
     const MaskGeom& geo = prm.geom;
     const int c0 = kt * kTile;
     long long rq_lo, rq_hi;
-    kv_tile_q_range(geo, c0, &rq_lo, &rq_hi);
+    const bool flagged = prm.heads.flag[slot] != 0;
+    kv_tile_q_range(geo, c0, flagged, &rq_lo, &rq_hi);
     const int qt_lo = (int)(rq_lo / kTile);
     const int n_qt = rq_hi >= rq_lo ? (int)(rq_hi / kTile) - qt_lo + 1 : 0;
     const int n_it = n_qt * prm.g;
@@ -630,7 +631,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
         const int jl = c0 + row;
         const long long jpos = (long long)geo.kv_pos0 + jl;
         // query rows that read this key differentiably: [qlo, qhi]
-        long long qlo_ll = jpos - geo.q_pos0, qhi_ll = hi_diff(geo, jpos < 0 ? 0 : jpos) - 1 - geo.q_pos0;
+        long long qlo_ll = jpos - geo.q_pos0, qhi_ll = hi_diff(geo, jpos < 0 ? 0 : jpos, flagged) - 1 - geo.q_pos0;
         if (jpos < 0) qhi_ll = -1;
         if (qlo_ll < 0) qlo_ll = 0;
         if (qhi_ll > geo.Lq - 1) qhi_ll = geo.Lq - 1;
@@ -638,7 +639,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
         // no element mask when every key row of the tile is read by every query row of the query tile
         const long long jfirst = (long long)geo.kv_pos0 + c0, jlast = jfirst + kTile - 1;
         const long long full_qlo = jlast - geo.q_pos0;  // latest first-reader
-        long long full_qhi = (jfirst >= 0 ? hi_diff(geo, jfirst) : 0) - 1 - geo.q_pos0;  // earliest last-reader
+        long long full_qhi = (jfirst >= 0 ? hi_diff(geo, jfirst, flagged) : 0) - 1 - geo.q_pos0;  // earliest last-reader
         if (full_qhi > geo.Lq - 1) full_qhi = geo.Lq - 1;
         const bool keys_in_range = c0 + kTile <= geo.kv_len && jfirst >= 0;
 

@@ -22,6 +22,7 @@ struct MaskGeom {
     int S, T;
     int q_pos0, kv_pos0;
     int Lq, kv_len;
+    int flagged_tail_sg;  // flagged heads read the carried tail forward-only too (Appendix C, Eq. "ctx", read literally)
 };
 
 // p / S for a non-negative position: positions fit 32 bits in practice, and a 32-bit division is
@@ -36,10 +37,15 @@ __host__ __device__ inline long long tail_start(const MaskGeom& g, long long p) 
 __host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, bool flagged) {
     return flagged ? 0 : tail_start(g, p);
 }
-// one past the last query position that differentiably reads key position j
-__host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j) {
+// one past the last query position that differentiably reads key position j (of a flagged head or not)
+__host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, bool flagged) {
     long long seg_end = (seg_of(j, g.S) + 1) * (long long)g.S;
+    if (flagged && g.flagged_tail_sg) return seg_end;
     return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
+}
+// first key position query position p reads differentiably
+__host__ __device__ inline long long lo_diff(const MaskGeom& g, long long p, bool flagged) {
+    return (flagged && g.flagged_tail_sg) ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
 }
 
 // Local key-row range [jl_lo, jl_hi] (inclusive) that the query tile starting at row r0 can see;
@@ -58,14 +64,14 @@ __host__ __device__ inline void q_tile_kv_range(const MaskGeom& g, int r0, bool 
 }
 // Query-row range [r_lo, r_hi] (inclusive) that differentiably reads some key of the key tile
 // starting at local row c0; empty when r_hi < r_lo.
-__host__ __device__ inline void kv_tile_q_range(const MaskGeom& g, int c0, long long* r_lo, long long* r_hi) {
+__host__ __device__ inline void kv_tile_q_range(const MaskGeom& g, int c0, bool flagged, long long* r_lo, long long* r_hi) {
     int c_last = c0 + kTile - 1;
     if (c_last > g.kv_len - 1) c_last = g.kv_len - 1;
     long long j0 = (long long)g.kv_pos0 + c0, j1 = (long long)g.kv_pos0 + c_last;
     if (j1 < 0) { *r_lo = 0; *r_hi = -1; return; }
     if (j0 < 0) j0 = 0;
     long long a = j0 - g.q_pos0;              // first query position is the key itself
-    long long b = hi_diff(g, j1) - 1 - g.q_pos0;  // hi_diff is non-decreasing in j
+    long long b = hi_diff(g, j1, flagged) - 1 - g.q_pos0;  // hi_diff is non-decreasing in j
     if (a < 0) a = 0;
     if (b > g.Lq - 1) b = g.Lq - 1;
     *r_lo = a;

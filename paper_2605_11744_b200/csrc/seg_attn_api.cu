@@ -81,6 +81,7 @@ bool params_ok(const seg_attn_params* p) {
     if (p->d != 64 && p->d != 128) return false;
     if (p->S < 1 || p->T < 0 || p->T > p->S) return false;
     if (p->q_pos0 < 0) return false;
+    if (p->flags & ~SEGATTN_FLAG_FLAGGED_TAIL_SG) return false;
     if (!(p->sm_scale > 0.f) || !std::isfinite(p->sm_scale)) return false;
     if ((long long)p->q_pos0 + p->Lq > 0x7fffffffLL / 2) return false;
     return true;
@@ -135,6 +136,7 @@ MaskGeom geom_of(const seg_attn_params* p) {
     g.kv_pos0 = p->kv_pos0;
     g.Lq = p->Lq;
     g.kv_len = p->kv_len;
+    g.flagged_tail_sg = (p->flags & SEGATTN_FLAG_FLAGGED_TAIL_SG) ? 1 : 0;
     return g;
 }
 
@@ -273,7 +275,7 @@ segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* hea
             const long long pos = (long long)g.q_pos0 + r;
             long long hi = pos - g.kv_pos0;
             if (hi > g.kv_len - 1) hi = g.kv_len - 1;
-            long long lo = lo_visible(g, pos, f) - g.kv_pos0, lod = tail_start(g, pos) - g.kv_pos0;
+            long long lo = lo_visible(g, pos, f) - g.kv_pos0, lod = lo_diff(g, pos, f) - g.kv_pos0;
             if (lo < 0) lo = 0;
             if (lod < 0) lod = 0;
             if (hi >= lo) v += hi - lo + 1;

@@ -105,6 +105,10 @@ def test_pair_counter_matches_oracle_enumeration(B, L, Hq, Hkv, S, T, mask):
     nv, nd, tiles = sa.count_pairs(B, L, Hq, Hkv, 128, S, T, mask)
     assert (nv, nd) == oracle.count_pairs(B, L, Hq, Hkv, S, T, mask)
     assert tiles * 128 * 128 >= nv
+    # the reading in which flagged heads read the carried tail forward-only too: fewer differentiable pairs
+    nv2, nd2, _ = sa.count_pairs(B, L, Hq, Hkv, 128, S, T, mask, flagged_tail_is_sg=True)
+    assert (nv2, nd2) == oracle.count_pairs(B, L, Hq, Hkv, S, T, mask, flagged_tail_is_sg=True)
+    assert nv2 == nv and nd2 <= nd
 
 
 def test_benchmark_configuration_counts():

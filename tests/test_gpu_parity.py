@@ -40,6 +40,28 @@ def test_small_cases_match_oracle_elementwise(B, L, Hq, Hkv, d, S, T, mask):
     assert_grads_close((dQ, dK, dV), ref, "bwd")
 
 
+@pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask", [
+    (1, 1024, 4, 2, 128, 256, 128, [0, 1]),
+    (2, 700, 4, 2, 128, 200, 72, [1, 0]),
+    (1, 640, 2, 2, 128, 64, 64, [1, 1]),
+    (1, 333, 2, 2, 64, 100, 100, [0, 1]),
+])
+def test_flagged_heads_reading_the_tail_forward_only(B, L, Hq, Hkv, d, S, T, mask):
+    # the literal reading of Eq. "ctx": only unflagged (local) heads send gradient through the carried tail
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=L + T)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask, flagged_tail_is_sg=True)
+    sa.poll_status()
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask, flagged_tail_is_sg=True)
+    assert_grads_close((dQ, dK, dV), ref, "flagged tail sg")
+    # it differs from the default reading exactly on the flagged heads' K/V gradients
+    dQ0, dK0, dV0 = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask)
+    assert torch.equal(dQ, dQ0)
+    for c, f in enumerate(mask):
+        same = torch.equal(dK[:, :, c], dK0[:, :, c]) and torch.equal(dV[:, :, c], dV0[:, :, c])
+        assert same == (not f or T == 0)
+
+
 def test_configuration_1_in_full():
     w = workloads.CONFIGS[0]
     x = workloads.make_inputs(w)
