@@ -191,6 +191,12 @@ segattn_status seg_attn_profile_kernels(const seg_attn_params* p, const void* Q,
                                        void* O, float* LSE, const void* dO, const uint8_t* head_past_mask, void* dQ,
                                        void* dK, void* dV, void* workspace, size_t workspace_bytes, int iters,
                                        float ms_per_launch[4], void* stream);
+/* Diagnostic aid (the paper has no counterpart): enqueues a one-warp kernel that waits, with a
+ * 1 ms limit, on a barrier nothing ever signals - the way every wait inside the library's kernels
+ * is bounded.  The wait gives up, the kernel ends normally, and the next seg_attn_poll_status
+ * returns SEGATTN_ERR_TIMEOUT (seg_attn_last_cuda_error() then gives (4 << 8) | 99) and clears
+ * the status word; the context stays usable. */
+segattn_status seg_attn_selftest_wait_timeout(void* stream);
 /* Number of kernel launches the library has enqueued so far in this process. */
 int64_t seg_attn_launch_count(void);
 

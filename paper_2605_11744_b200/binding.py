@@ -62,6 +62,7 @@ def lib():
         L.seg_attn_profile_kernels.argtypes = [pp, vp, vp, vp, vp, fp, vp, u8p, vp, vp, vp, vp, ctypes.c_size_t,
                                                ctypes.c_int, ctypes.POINTER(ctypes.c_float * 4), vp]
         L.seg_attn_poll_status.argtypes = [vp]
+        L.seg_attn_selftest_wait_timeout.argtypes = [vp]
         L.seg_attn_status_string.restype = ctypes.c_char_p
         L.seg_attn_status_string.argtypes = [ctypes.c_int]
         L.seg_attn_last_cuda_error.restype = ctypes.c_int
@@ -276,6 +277,12 @@ class Prefill:
 
 def poll_status(stream=None):
     _check(lib().seg_attn_poll_status(_stream(stream)), "seg_attn_poll_status")
+
+
+def selftest_wait_timeout(stream=None):
+    """Enqueue the kernel whose bounded wait runs out (C entry point `seg_attn_selftest_wait_timeout`);
+    the next `poll_status` raises SegAttnError with status 4."""
+    _check(lib().seg_attn_selftest_wait_timeout(_stream(stream)), "seg_attn_selftest_wait_timeout")
 
 
 def launch_count() -> int:

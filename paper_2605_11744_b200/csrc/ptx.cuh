@@ -66,13 +66,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Waits for the phase with the given parity to complete.  Gives up (returns false) when the
 // library's status word is already set by someone else, or after kWaitLimitNs, in which case
 // it records `site` in the status word.  Callers leave their loops on false.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int site) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int site,
+                                            unsigned long long limit_ns = kWaitLimitNs) {
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0) {
             if (*reinterpret_cast<volatile int*>(&g_device_status) != 0) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            if (global_ns() - t0 > limit_ns) {
                 atomicCAS(&g_device_status, 0, (4 << 8) | (site & 0xff));
                 return false;
             }

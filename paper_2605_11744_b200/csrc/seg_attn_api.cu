@@ -301,6 +301,28 @@ segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* hea
 #include "seg_attn_bwd_api.inc"
 #include "seg_attn_prefill_api.inc"
 
+// ---- Self-test of the bounded waits ------------------------------------------------------------
+namespace {
+// One warp waits on an mbarrier nobody arrives on, with a 1 ms limit: the wait gives up, records
+// site 99 in the status word and the kernel returns normally.
+__global__ void selftest_wait_kernel() {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) mbar_wait_slow(smem_u32(&bar), 0, 99, 1000000ull);
+}
+}  // namespace
+
+extern "C" segattn_status seg_attn_selftest_wait_timeout(void* stream) {
+    segattn_status st = check_arch();
+    if (st != SEGATTN_OK) return st;
+    selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+    return launch_check();
+}
+
 // ---- Backward without a caller-provided workspace ---------------------------------------------
 // The row dots D = <dO, O> of seg_attn_bwd_static live here instead of in caller memory.  In host
 // code this name is only a handle for the runtime's symbol calls, never a device address: the

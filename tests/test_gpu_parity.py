@@ -222,3 +222,18 @@ def test_host_buffer_step_matches_device_path():
     dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, w.S, w.T, x["mask"], w.sm_scale)
     for k, t in (("O", O), ("LSE", LSE), ("dQ", dQ), ("dK", dK), ("dV", dV)):
         assert torch.equal(outs[k], t.cpu()), k
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
+    # a wait on a barrier nothing signals gives up after its limit and sets the status word: no hang, no fault
+    sa.poll_status()
+    sa.selftest_wait_timeout()
+    with pytest.raises(sa.SegAttnError) as e:
+        sa.poll_status()
+    assert e.value.status == 4
+    assert sa.lib().seg_attn_last_cuda_error() == (4 << 8) | 99
+    sa.poll_status()   # the word was cleared
+    Q, K, V, dO = rand_inputs(1, 256, 2, 1, 128, seed=2)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, 128, 64, [0])
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), 128, 64, [0])
+    assert_fwd_close(O, LSE, Oo, LSEo, "after a timeout")
