@@ -366,6 +366,37 @@ def run_ours(args, w):
         print(json.dumps(line), flush=True)
 
 
+def run_table(args):
+    """One JSON line per workload (configurations 1-3 and the 24 points of sweep 5): per-kernel CUDA-event
+    times with inputs resident in HBM, and the throughput over unmasked work they give.  Fills the
+    results table of the benchmark spec; not the benchmark line."""
+    import paper_2605_11744_b200 as sa
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    for w in list(workloads.CONFIGS[:3]) + workloads.sweep():
+        x = workloads.make_inputs(w, device="cuda")
+        fm = flop_model(w, x["mask"], sa.count_pairs)
+        per = sa.profile_kernels(x["Q"], x["K"], x["V"], x["dO"], w.S, w.T, x["mask"], w.sm_scale, iters=max(3, min(args.steps, 10)))
+        sa.poll_status()
+        bwd_ms = per["rowdot"] + per["dq"] + per["dkv"]
+        tot_ms = per["fwd"] + bwd_ms
+        tf = lambda flops, ms: flops / (ms / 1e3) / 1e12
+        print(json.dumps({
+            "workload": w.name, "B": w.B, "L": w.L, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "S": w.S, "T": w.T,
+            "past_frac": w.past_frac, "pairs_visible": fm["pairs_visible"], "pairs_diff": fm["pairs_diff"],
+            "tflop_fwd": fm["fwd"] / 1e12, "tflop_bwd": fm["bwd"] / 1e12,
+            "ms": {k: round(per[k], 4) for k in ("fwd", "rowdot", "dq", "dkv")},
+            "tflops_fwd": tf(fm["fwd"], per["fwd"]), "tflops_bwd": tf(fm["bwd"], bwd_ms),
+            "tflops_total": tf(fm["fwd"] + fm["bwd"], tot_ms),
+            "frac_of_bf16_peak": tf(fm["fwd"] + fm["bwd"], tot_ms) / peaks["bf16"],
+            "frac_of_bf16_sustained": tf(fm["fwd"] + fm["bwd"], tot_ms) / peaks["bf16_sustained"],
+            "issued_over_algorithmic_fwd": fm["fwd_issued"] / fm["fwd"]}), flush=True)
+        del x
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -374,7 +405,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="benchmark configuration number (1-5); default 2")
     ap.add_argument("--no-prefill", action="store_true", help="skip the configuration-4 streamed prefill measurement")
+    ap.add_argument("--table", action="store_true",
+                    help="per-kernel timings of configurations 1-3 and the sweep, one JSON line each (not the benchmark line)")
     args = ap.parse_args()
+    if args.table:
+        run_table(args)
+        return
     w = workloads.CONFIGS[args.config - 1]
     if args.impl == "reference":
         run_reference(args, w)
