@@ -62,6 +62,28 @@ def test_flagged_heads_reading_the_tail_forward_only(B, L, Hq, Hkv, d, S, T, mas
         assert same == (not f or T == 0)
 
 
+def test_window_of_queries_with_position_offsets():
+    # queries of segments 2..3 only (q_pos0 = 2 S) against all keys up to their end: forward and backward
+    # equal the oracle's for the same window; this is the call shape of a windowed training step
+    B, L, Hq, Hkv, d, S, T = 1, 1024, 4, 2, 128, 256, 128
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=17)
+    mask = [1, 0]
+    q0, q1 = 2 * S, 4 * S
+    Qw, dOw, Kw, Vw = Q[:, q0:q1].contiguous(), dO[:, q0:q1].contiguous(), K[:, :q1].contiguous(), V[:, :q1].contiguous()
+    O, LSE = sa.seg_attn_fwd(Qw, Kw, Vw, S, T, mask, q_pos0=q0)
+    dQ, dK, dV = sa.seg_attn_bwd(Qw, Kw, Vw, O, LSE, dOw, S, T, mask, q_pos0=q0)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Qw), f64(Kw), f64(Vw), S, T, mask, q_pos0=q0)
+    ref = oracle.bwd(f64(Qw), f64(Kw), f64(Vw), f64(dOw), S, T, mask, q_pos0=q0)
+    assert_fwd_close(O, LSE, Oo, LSEo, "window")
+    assert_grads_close((dQ, dK, dV), ref, "window")
+    # keys before the tail of segment 1 get gradient from no query of the window
+    assert torch.count_nonzero(dK[:, :q0 - T]) == 0 and torch.count_nonzero(dV[:, :q0 - T]) == 0
+    # the forward of the window equals the rows of the whole-sequence forward, bit for bit (same tiles)
+    O_all, LSE_all = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    assert torch.equal(O, O_all[:, q0:q1]) and torch.equal(LSE, LSE_all[:, :, q0:q1])
+
+
 def test_configuration_1_in_full():
     w = workloads.CONFIGS[0]
     x = workloads.make_inputs(w)
