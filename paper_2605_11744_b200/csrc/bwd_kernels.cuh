@@ -141,6 +141,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
     using SM = DqSmem<D>;
     constexpr int trace_id = 1;
     (void)trace_id;
+    TRACE_INIT();
     constexpr int NK = SM::kKStages, NV = SM::kVStages;
     enum { kBarQFull = 0, kBarQEmpty, kBarDoFull, kBarDoEmpty, kBarKFull, kBarKEmpty = kBarKFull + NK,
            kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV, kBarSFull = kBarVEmpty + NV, kBarDpFull = kBarSFull + 2,
@@ -221,7 +222,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
         constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
         constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
         int qn = 0;
-        long long g = 0;  // key tiles of earlier work items
+        int g = 0;  // key tiles of earlier work items (a CTA sees far fewer than 2^31)
         bool ok = true;
         ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items_dq);
         for (int item; ok && walk.next(&item);) {
@@ -230,55 +231,65 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
             dq_item_tiles(prm, it, &t_lo, &n);
             if (n == 0) continue;
             // Waits on tiles brought by TMA need no tcgen05 fence.
-            auto wait_k = [&](int j) { return warp_wait(bar(kBarKFull + (int)((g + j) % NK)), (uint32_t)(((g + j) / NK) & 1), 14); };
-            auto wait_v = [&](int j) { return warp_wait(bar(kBarVFull + (int)((g + j) % NV)), (uint32_t)(((g + j) / NV) & 1), 15); };
+            auto wait_k = [&](int j) { return warp_wait(bar(kBarKFull + (g + j) % NK), (uint32_t)((g + j) / NK) & 1, 14); };
+            auto wait_v = [&](int j) { return warp_wait(bar(kBarVFull + (g + j) % NV), (uint32_t)((g + j) / NV) & 1, 15); };
             auto issue_s = [&](int j) {   // S(j) = Q K_j^T into the S buffer of the tile's global parity
-                const long long gj = g + j;
-                const int sk = (int)(gj % NK);
+                const int gj = g + j;
+                const uint64_t qd = make_sdesc(sQ, 16, 1024), kd = make_sdesc(sK(gj % NK), 16, 1024);
+                const uint32_t d_s = tS0 + (uint32_t)(gj & 1) * 128;
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-                    mma_ss(tS0 + (uint32_t)(gj & 1) * 128, make_sdesc(sQ + off, 16, 1024), make_sdesc(sK(sk) + off, 16, 1024),
-                           idesc_s, k > 0);
+                    const uint32_t off = ((k / 4) * 16384 + (k % 4) * 32) >> 4;  // descriptor addresses count 16-byte units
+                    mma_ss(d_s, qd + off, kd + off, idesc_s, k > 0);
                 }
-                mma_commit(bar(kBarSFull + (int)(gj & 1)));
-                if (j == n - 1) mma_commit(bar(kBarQEmpty));   // the item's last scores release Q
+                mma_commit(bar(kBarSFull + (gj & 1)));
+                mma_commit_if(j == n - 1, bar(kBarQEmpty));   // the item's last scores release Q
             };
             auto issue_dp = [&](int j) {  // dP(j) = dO V_j^T
-                const int sv = (int)((g + j) % NV);
+                const int sv = (g + j) % NV;
+                const uint64_t od = make_sdesc(sDO, 16, 1024), vd = make_sdesc(sV(sv), 16, 1024);
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-                    mma_ss(tDp, make_sdesc(sDO + off, 16, 1024), make_sdesc(sV(sv) + off, 16, 1024), idesc_s, k > 0);
+                    const uint32_t off = ((k / 4) * 16384 + (k % 4) * 32) >> 4;
+                    mma_ss(tDp, od + off, vd + off, idesc_s, k > 0);
                 }
                 mma_commit(bar(kBarVEmpty + sv));
                 mma_commit(bar(kBarDpFull));
             };
-            ok = warp_wait(bar(kBarQFull), qn & 1, 13) && wait_k(0);
+            ok = warp_wait2(bar(kBarQFull), qn & 1, bar(kBarKFull + g % NK), (uint32_t)(g / NK) & 1, 13);
             if (ok) issue_s(0);
-            ok = ok && warp_wait(bar(kBarDoFull), qn & 1, 13) && wait_v(0);
+            ok = ok && warp_wait2(bar(kBarDoFull), qn & 1, bar(kBarVFull + g % NV), (uint32_t)(g / NV) & 1, 13);
             if (ok) issue_dp(0);
             if (ok && n > 1 && (ok = wait_k(1))) issue_s(1);
+            // The loop is bound by the latency of its own control flow between the batches of products:
+            // what a run needs at its start is polled together (one vote, one branch when all of it is
+            // there, as it usually is), and optional completion signals are predicated.
             for (int j = 0; ok && j < n; ++j) {
-                const long long gj = g + j;
-                if (j + 1 < n) ok = wait_v(j + 1);
-                ok = ok && warp_wait(bar(kBarDsFull), (uint32_t)(gj & 1), 16);   // dS(j) written, dP(j) read
-                if (!ok) break;
+                const int gj = g + j;
+                const bool has1 = j + 1 < n;
+                // V(j+1) landed (if there is one); dS(j) written and dP(j) read
+                const bool ready = (!has1 | mbar_test_wait(bar(kBarVFull + (gj + 1) % NV), (uint32_t)((gj + 1) / NV) & 1)) &
+                                   mbar_test_wait(bar(kBarDsFull), (uint32_t)(gj & 1));
+                if (!__all_sync(0xffffffffu, ready)) {
+                    ok = (!has1 || wait_v(j + 1)) && warp_wait(bar(kBarDsFull), (uint32_t)(gj & 1), 16);
+                    if (!ok) break;
+                }
                 tc_fence_after();
                 TRACE(lane == 0, j * 16 + 4);
-                if (j + 1 < n) issue_dp(j + 1);   // first: phase B of the next tile waits for it
-                const int sk = (int)(gj % NK);
+                if (has1) issue_dp(j + 1);   // first: phase B of the next tile waits for it
+                const int sk = gj % NK;
+                const uint32_t a_ds = tS0 + (uint32_t)(gj & 1) * 128;
+                const uint64_t kd = make_sdesc(sK(sk), 16384, 1024);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tDq, tS0 + (uint32_t)(gj & 1) * 128 + packed_a_col(k), make_sdesc(sK(sk) + k * 2048, 16384, 1024),
-                           idesc_dq, (j > 0) || (k > 0));
+                    mma_ts(tDq, a_ds + packed_a_col(k), kd + ((k * 2048) >> 4), idesc_dq, (j > 0) || (k > 0));
                 mma_commit(bar(kBarKEmpty + sk));
+                mma_commit_if(j == n - 1, bar(kBarDqFull));
                 // K(j+2) reuses the stage dQ(j-1) released one run ago: its load gets the first two products
                 // of this run as extra time before it is waited for
                 if (j + 2 < n && (ok = wait_k(j + 2))) issue_s(j + 2);    // overwrites dS(j): after dQ(j)
                 TRACE(lane == 0, j * 16 + 5);
             }
-            if (ok) mma_commit(bar(kBarDqFull));
             ++qn;
             g += n;
         }
@@ -479,6 +490,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
     using SM = DkvSmem<D>;
     constexpr int trace_id = 2;
     (void)trace_id;
+    TRACE_INIT();
     constexpr int NS = SM::kStages;
     enum { kBarKV = 0, kBarQFull = 1, kBarQEmpty = kBarQFull + NS, kBarDoFull = kBarQEmpty + NS,
            kBarDoEmpty = kBarDoFull + NS, kBarSFull = kBarDoEmpty + NS, kBarDpFull, kBarPFull, kBarDsFull, kBarDone,

@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     using SM = FwdSmem<D>;
     constexpr int trace_id = 0;
     (void)trace_id;
+    TRACE_INIT();
     constexpr int NQ = SM::kQStages, NK = SM::kKStages, NV = SM::kVStages;
     enum { kBarQFull = 0, kBarQEmpty = kBarQFull + NQ, kBarKFull = kBarQEmpty + NQ, kBarKEmpty = kBarKFull + NK,
            kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV, kBarSFull = kBarVEmpty + NV, kBarPFull = kBarSFull + 3,

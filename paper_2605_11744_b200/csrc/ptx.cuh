@@ -18,8 +18,11 @@ __device__ int g_device_status = 0;
 __device__ long long g_trace[4096];
 __device__ int g_trace_block = 0;
 __device__ int g_trace_kernel = 0;
-#define TRACE(cond, idx) do { if ((cond) && blockIdx.x == g_trace_block && g_trace_kernel == trace_id && (idx) < 4096) { long long t_; asm volatile("mov.u64 %0, %clock64;" : "=l"(t_)); g_trace[(idx)] = t_; } } while (0)
+// TRACE_INIT reads the selection once per thread, so that a stamp costs a clock read and a store.
+#define TRACE_INIT() const bool trace_on_ = (blockIdx.x == g_trace_block && g_trace_kernel == trace_id)
+#define TRACE(cond, idx) do { if (trace_on_ && (cond) && (idx) < 4096) { long long t_; asm volatile("mov.u64 %0, %clock64;" : "=l"(t_)); g_trace[(idx)] = t_; } } while (0)
 #else
+#define TRACE_INIT() do { } while (0)
 #define TRACE(cond, idx) do { } while (0)
 #endif
 
@@ -57,6 +60,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Non-blocking test of the same condition (try_wait may suspend the thread for a while first).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -239,9 +254,30 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
         "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
         : "memory");
 }
+// The same, only if `pred` (warp-uniform) holds: a predicated instruction instead of a branch.
+__device__ __forceinline__ void mma_commit_if(bool pred, uint32_t bar) {
+    asm volatile(
+        "{\n\t.reg .pred q, r;\n\telect.sync _|q, 0xffffffff;\n\tsetp.ne.b32 r, %1, 0;\n\tand.pred q, q, r;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar),
+        "r"((uint32_t)pred)
+        : "memory");
+}
 // A bounded wait executed by a whole warp, with a warp-uniform result.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, int site) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, site));
+}
+// Bounded waits of a whole warp on two or three barriers at once: one poll of each, one vote and
+// one branch when all of them have completed already, which is the common case for an MMA issuer.
+__device__ __forceinline__ bool warp_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b, int site) {
+    const bool done = mbar_try_wait(bar_a, par_a) & mbar_try_wait(bar_b, par_b);
+    if (__all_sync(0xffffffffu, done)) return true;
+    return warp_wait(bar_a, par_a, site) && warp_wait(bar_b, par_b, site);
+}
+__device__ __forceinline__ bool warp_wait3(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b, uint32_t bar_c,
+                                           uint32_t par_c, int site) {
+    const bool done = mbar_try_wait(bar_a, par_a) & mbar_try_wait(bar_b, par_b) & mbar_try_wait(bar_c, par_c);
+    if (__all_sync(0xffffffffu, done)) return true;
+    return warp_wait(bar_a, par_a, site) && warp_wait(bar_b, par_b, site) && warp_wait(bar_c, par_c, site);
 }
 
 // ---- small numeric helpers ---------------------------------------------------------------------
