@@ -75,8 +75,8 @@ def _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg):
 
 def _mask(head_past_mask, Hkv):
     m = np.zeros(Hkv, dtype=np.uint8) if head_past_mask is None else \
-        np.ascontiguousarray(np.asarray(head_past_mask) != 0, dtype=np.uint8)
-    assert m.shape == (Hkv,)
+        np.ascontiguousarray(np.asarray(head_past_mask), dtype=np.uint8)  # head class: 0 local, 1 past, 2 own only
+    assert m.shape == (Hkv,) and int(m.max(initial=0)) <= 2
     return m
 
 

@@ -5,7 +5,8 @@ that the two can be checked against each other and against library attention:
 
 * ``visible[p, j] = (j <= p) & ((j >= a[p]) | flag)`` with ``a[p] = max(0, (p // S) * S - T)``
   (own segment causally, the previous segment's last T positions, and - for a flagged KV head -
-  everything older; Appendix C, Eqs. "attn" and "ctx"; C_0 empty, Section 3.1);
+  everything older; Appendix C, Eqs. "attn" and "ctx"; C_0 empty, Section 3.1); a head of class 2
+  reads its own segment only, ``j >= (p // S) * S`` (third case of Eq. "ctx");
 * ``diff[p, j] = (j <= p) & (j >= a[p])``: the reads that carry gradient into K/V; older reads
   of a flagged head are stop-gradient (Definition 3.2, Lemma B.1).
 
@@ -22,8 +23,10 @@ def masks(Lq, Lk, S, T, flag, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False):
     seg0 = (p // S) * S
     a = np.maximum(0, seg0 - T)
     causal = j <= p
-    visible = causal & ((j >= a) | bool(flag))
-    lo_diff = seg0 if (flag and flagged_tail_is_sg) else a
+    cls = int(flag)  # head class: 0 local, 1 past access, 2 own segment only
+    lo_vis = {0: a, 1: np.zeros_like(a), 2: seg0}[cls]
+    visible = causal & (j >= lo_vis)
+    lo_diff = seg0 if (cls == 2 or (cls == 1 and flagged_tail_is_sg)) else a
     diff = causal & (j >= lo_diff)
     return visible, diff
 
@@ -34,7 +37,7 @@ def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0):
     _, Lk, Hkv, _ = K.shape
     g = Hq // Hkv
     scale = 1.0 / np.sqrt(d) if scale is None else scale
-    flags = np.zeros(Hkv, bool) if head_past_mask is None else np.asarray(head_past_mask) != 0
+    flags = np.zeros(Hkv, int) if head_past_mask is None else np.asarray(head_past_mask).astype(int)
     O = np.zeros_like(Q)
     LSE = np.full((B, Hq, Lq), -np.inf)
     for h in range(Hq):
@@ -57,7 +60,7 @@ def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0,
     _, Lk, Hkv, _ = K.shape
     g = Hq // Hkv
     scale = 1.0 / np.sqrt(d) if scale is None else scale
-    flags = np.zeros(Hkv, bool) if head_past_mask is None else np.asarray(head_past_mask) != 0
+    flags = np.zeros(Hkv, int) if head_past_mask is None else np.asarray(head_past_mask).astype(int)
     dQ, dK, dV = np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V)
     for h in range(Hq):
         c = h // g

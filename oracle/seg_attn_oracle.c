@@ -23,6 +23,10 @@
  *     start, dense (no top-k retrieval), in union with the tail and the own
  *     segment.  With flagged_tail_is_sg != 0 the flagged head's tail reads are
  *     stop-gradient too (the variant where only local heads carry the state).
+ *   - head_past_mask[c] is a head class: 0 local, 1 flagged as above, 2 a head
+ *     whose context is its own segment alone (the long-range head of a layer
+ *     outside the long-range layers, Appendix C, Eq. "ctx", third case):
+ *     visible = diff = { i*S <= j <= p }.
  *
  * Global positions: query row r sits at p = q_pos0 + r, key row jl at
  * j = kv_pos0 + jl.  With i = p / S and a_i = max(0, i*S - T):
@@ -73,6 +77,10 @@ static void row_bounds(const oracle_cfg *c, int flag, long p, long *lo_vis, long
     long i = p / c->S;
     long a = i * (long)c->S - c->T;
     if (a < 0) a = 0;
+    if (flag == 2) {             /* own segment only (Appendix C, Eq. "ctx", third case) */
+        *lo_vis = *lo_diff = i * (long)c->S;
+        return;
+    }
     *lo_vis = flag ? 0 : a;
     *lo_diff = (flag && c->flagged_tail_is_sg) ? i * (long)c->S : a;
 }
@@ -138,7 +146,7 @@ int oracle_seg_attn_fwd(const oracle_cfg *c, const double *Q, const double *K, c
             int b = (int)(idx / ((long)c->Lq * c->Hq));
             int kvh = h / g;
             long p = (long)c->q_pos0 + r, lo_vis, lo_diff, j0, j1;
-            row_bounds(c, head_past_mask[kvh] != 0, p, &lo_vis, &lo_diff);
+            row_bounds(c, head_past_mask[kvh], p, &lo_vis, &lo_diff);
             local_range(c, lo_vis, p, &j0, &j1);
             const double *q = Q + (((long)b * c->Lq + r) * c->Hq + h) * d;
             double *o = O + (((long)b * c->Lq + r) * c->Hq + h) * d;
@@ -189,7 +197,7 @@ int oracle_seg_attn_bwd(const oracle_cfg *c, const double *Q, const double *K, c
             int b = (int)(idx / ((long)c->Lq * c->Hq));
             int kvh = h / g;
             long p = (long)c->q_pos0 + r, lo_vis, lo_diff, j0, j1;
-            row_bounds(c, head_past_mask[kvh] != 0, p, &lo_vis, &lo_diff);
+            row_bounds(c, head_past_mask[kvh], p, &lo_vis, &lo_diff);
             local_range(c, lo_vis, p, &j0, &j1);
             const double *Kb = K + (long)b * c->Lk * c->Hkv * d;
             const double *Vb = V + (long)b * c->Lk * c->Hkv * d;
@@ -228,7 +236,7 @@ int oracle_seg_attn_bwd(const oracle_cfg *c, const double *Q, const double *K, c
         long jl = (idx / c->Hkv) % c->Lk;
         int b = (int)(idx / ((long)c->Hkv * c->Lk));
         long j = (long)c->kv_pos0 + jl;
-        int flag = head_past_mask[kvh] != 0;
+        int flag = head_past_mask[kvh];
         const double *k = K + (((long)b * c->Lk + jl) * c->Hkv + kvh) * d;
         const double *v = V + (((long)b * c->Lk + jl) * c->Hkv + kvh) * d;
         double *gk = dK + (((long)b * c->Lk + jl) * c->Hkv + kvh) * d;
@@ -271,7 +279,7 @@ int oracle_count_pairs(const oracle_cfg *c, const uint8_t *head_past_mask,
     const int g = c->Hq / c->Hkv;
     int64_t nv = 0, nd = 0;
     for (int h = 0; h < c->Hq; ++h) {
-        int flag = head_past_mask[h / g] != 0;
+        int flag = head_past_mask[h / g];
         for (long r = 0; r < c->Lq; ++r) {
             long p = (long)c->q_pos0 + r, lo_vis, lo_diff, j0, j1;
             row_bounds(c, flag, p, &lo_vis, &lo_diff);

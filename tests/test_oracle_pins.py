@@ -79,6 +79,32 @@ def test_all_heads_flagged_forward_is_full_causal(S, T):
 
 
 # ---- the paper's segment recurrence, built with library ops and autograd -----------------------
+def test_own_segment_only_heads_are_block_diagonal_for_any_tail():
+    # A head of class 2 never reads the carried tail: for any T it equals T = 0, i.e. independent
+    # causal attention per segment (Appendix C, Eq. "ctx", third case), in values and gradients.
+    S, L, T = 24, 96, 11
+    Q, K, V, dO = rand(1, L, 4, 2, 8)
+    O, LSE = oracle.fwd(Q, K, V, S, T, head_past_mask=[2, 0])
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=[2, 0])
+    hq, c = slice(0, 2), slice(0, 1)
+    for i in range(L // S):
+        sl = slice(i * S, (i + 1) * S)
+        o, lse, gq, gk, gv = sdpa_causal(Q[:, sl, hq], K[:, sl, c], V[:, sl, c], dO[:, sl, hq])
+        np.testing.assert_allclose(O[:, sl, hq], o, atol=TOL)
+        np.testing.assert_allclose(LSE[:, hq, sl], lse, atol=TOL)
+        np.testing.assert_allclose(dQ[:, sl, hq], gq, atol=TOL)
+        np.testing.assert_allclose(dK[:, sl, c], gk, atol=TOL)
+        np.testing.assert_allclose(dV[:, sl, c], gv, atol=TOL)
+    # the local head beside it is untouched by its neighbour's class
+    O0, _ = oracle.fwd(Q, K, V, S, T, head_past_mask=[0, 0])
+    np.testing.assert_array_equal(O[:, :, 2:], O0[:, :, 2:])
+    # and the dense statement of the definition agrees
+    d2 = dense.bwd(Q, K, V, dO, S, T, head_past_mask=[2, 0])
+    for a, b in zip((dQ, dK, dV), d2):
+        np.testing.assert_allclose(a, b, atol=TOL)
+    np.testing.assert_allclose(dense.fwd(Q, K, V, S, T, head_past_mask=[2, 0])[0], O, atol=TOL)
+
+
 def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False):
     """For every segment i and head: context = [sg(older past) if flagged ; tail of segment i-1 ;
     own segment], every prefix position visible and the own segment causal (Appendix C), run
@@ -96,12 +122,12 @@ def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False):
         for h in range(Hq):
             c = h // g
             ks, vs = [], []
-            if flags[c] and a > 0:
+            if flags[c] == 1 and a > 0:
                 ks.append(k[:, :a, c].detach())
                 vs.append(v[:, :a, c].detach())
-            if s0 > a:
+            if flags[c] != 2 and s0 > a:      # class 2: the own segment is the whole context
                 kt, vt = k[:, a:s0, c], v[:, a:s0, c]
-                if flags[c] and flagged_tail_is_sg:
+                if flags[c] == 1 and flagged_tail_is_sg:
                     kt, vt = kt.detach(), vt.detach()
                 ks.append(kt)
                 vs.append(vt)
@@ -128,6 +154,9 @@ def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False):
     (90, 30, 7, [1, 1], False),
     (96, 32, 8, [0, 1], True),        # flagged heads' tail reads stop-gradient too
     (64, 16, 0, [0, 0], False),
+    (96, 32, 8, [2, 0], False),       # an own-segment-only head beside a local one
+    (100, 32, 8, [1, 2], False),      # ... beside a past-access one, ragged last segment
+    (96, 32, 32, [2, 2], True),
 ])
 def test_segment_recurrence_with_autograd(L, S, T, flags, variant):
     Q, K, V, dO = rand(2, L, 4, 2, 8)
@@ -266,6 +295,9 @@ def test_pair_counts_match_closed_forms(L, S, T):
     assert nv == 2 * 2 * (local + full) and nd == 2 * 4 * local
     nv, nd = oracle.count_pairs(1, L, 4, 4, S, T)
     assert nv == nd == 4 * local
+    own = N * S * (S + 1) // 2                       # class 2: the causal triangle of each segment
+    nv, nd = oracle.count_pairs(1, L, 4, 2, S, T, head_past_mask=[2, 1])
+    assert nv == 2 * (own + full) and nd == 2 * (own + local)
 
 
 def test_benchmark_pair_counts():
