@@ -10,12 +10,15 @@
  *   - the carried KV tail: the last T key/value positions of the immediately preceding
  *     segment, the only differentiable cross-segment state (Section 3.4, "Local Continuity
  *     Channel"); the first segment has no carried state (Section 3.1, C_0 empty);
- *   - for KV heads flagged in `head_past_mask`, additionally every older key/value, read
- *     forward-only: stop-gradient, no gradient reaches those K/V (Definition 3.2; Section 3.4,
- *     "Long-Range Channel"; Appendix B, Lemma B.1).
+ *   - for KV heads of class SEGATTN_HEAD_PAST in `head_past_mask`, additionally every older
+ *     key/value, read forward-only: stop-gradient, no gradient reaches those K/V (Definition 3.2;
+ *     Section 3.4, "Long-Range Channel"; Appendix B, Lemma B.1);
+ *   - KV heads of class SEGATTN_HEAD_OWN read their own segment and nothing else: the context of
+ *     a long-range head in a layer that is not a long-range layer (Appendix C, Eq. "ctx", third
+ *     case).
  * With global positions p (query) and j (key), i = p / S and a_i = max(0, i*S - T):
- *     visible(p, j, c) <=> j <= p and (j >= a_i or head_past_mask[c] != 0)
- *     diff(p, j)       <=> a_i <= j <= p            (reads that carry gradient into K/V)
+ *     visible(p, j, c) <=> lo_c(p) <= j <= p,  lo_c(p) = a_i (LOCAL), 0 (PAST), i*S (OWN)
+ *     diff(p, j, c)    <=> max(lo_c(p), a_i) <= j <= p   (reads that carry gradient into K/V)
  * Query head h uses KV head c = h / (Hq / Hkv).
  *
  * Conventions that hold for every entry point unless it says otherwise:
@@ -23,8 +26,9 @@
  *     reallocates them.  Q, O, dO, dQ are bf16 [B][Lq][Hq][d]; K, V, dK, dV are bf16
  *     [B][kv_len][Hkv][d]; addressing is by the element strides in seg_attn_params (the last
  *     dimension is contiguous).  LSE is fp32, contiguous [B][Hq][Lq].
- *   - `head_past_mask` is a HOST array of Hkv bytes (non-zero = flagged); it is read before
- *     the call returns.
+ *   - `head_past_mask` is a HOST array of Hkv bytes, one head class per KV head (0 = local,
+ *     1 = past access, 2 = own segment only; any other value is SEGATTN_ERR_INVALID); it is read
+ *     before the call returns.
  *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it; no entry point
  *     synchronises the device except where stated.
  *   - Errors are return codes.  Arguments are validated on the host before anything is
@@ -55,6 +59,11 @@ typedef enum {
     SEGATTN_ERR_WORKSPACE = 5,        /* workspace/state buffer missing, misaligned or too small */
     SEGATTN_ERR_TOO_LARGE = 6         /* problem exceeds the fixed scratch of seg_attn_bwd_static */
 } segattn_status;
+
+/* Head classes, the entries of `head_past_mask` (Appendix C, Eq. "ctx"). */
+#define SEGATTN_HEAD_LOCAL 0 /* own segment + carried tail, both differentiable */
+#define SEGATTN_HEAD_PAST 1  /* own segment + carried tail + every older position (forward-only) */
+#define SEGATTN_HEAD_OWN 2   /* own segment only */
 
 /* seg_attn_params.flags, bit 0: for flagged KV heads the reads of the carried tail are stop-gradient
  * too, i.e. diff(p, j) <=> i*S <= j <= p for them.  This is the literal reading of Appendix C,

@@ -78,8 +78,9 @@ def _check(status: int, where: str):
 
 
 def _mask_arr(head_past_mask, Hkv: int) -> np.ndarray:
+    # one head class per KV head (booleans count as 0 / 1); the library rejects values above HEAD_OWN
     m = np.zeros(Hkv, dtype=np.uint8) if head_past_mask is None else \
-        np.ascontiguousarray(np.asarray(head_past_mask) != 0, dtype=np.uint8)
+        np.ascontiguousarray(np.asarray(head_past_mask), dtype=np.uint8)
     if m.shape != (Hkv,):
         raise ValueError("head_past_mask must have Hkv entries")
     return m
@@ -92,6 +93,7 @@ def _strides3(t: torch.Tensor):
 
 
 FLAG_FLAGGED_TAIL_SG = 1   # SEGATTN_FLAG_FLAGGED_TAIL_SG of the C header
+HEAD_LOCAL, HEAD_PAST, HEAD_OWN = 0, 1, 2   # SEGATTN_HEAD_* of the C header: entries of head_past_mask
 
 
 def params_for(Q, K, V, O, S: int, T: int, sm_scale: Optional[float] = None, q_pos0: int = 0,

@@ -94,7 +94,7 @@ struct DqSmem {
 
 struct DqItem {
     int b, hq, slot, qt;
-    bool flagged;
+    int cls;  // head class of the item's KV head
 };
 __device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) {
     const HeadTable& ht = prm.heads;
@@ -120,14 +120,14 @@ __device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) {
     it.slot = ht.order[cls_off + t % cls_n];
     it.b = t / cls_n;
     it.hq = ht.logical[it.slot] * prm.g + r;
-    it.flagged = ht.flag[it.slot] != 0;
+    it.cls = ht.flag[it.slot];
     return it;
 }
 
 // first visible key tile and number of visible key tiles of a work item of the dQ pass
 __device__ __forceinline__ void dq_item_tiles(const BwdParams& prm, const DqItem& it, int* t_lo, int* n_tiles) {
     long long jl_lo, jl_hi;
-    q_tile_kv_range(prm.geom, it.qt * kTile, it.flagged, false, &jl_lo, &jl_hi);
+    q_tile_kv_range(prm.geom, it.qt * kTile, it.cls, false, &jl_lo, &jl_hi);
     *t_lo = (int)(jl_lo / kTile);
     *n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - *t_lo + 1 : 0;
 }
@@ -313,12 +313,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
             const int r0 = it.qt * kTile;
             const int r = r0 + row;
             const long long p = (long long)geo.q_pos0 + r;
-            long long vlo_ll = lo_visible(geo, p, it.flagged) - geo.kv_pos0;
+            long long vlo_ll = lo_visible(geo, p, it.cls) - geo.kv_pos0;
             long long vhi_ll = p - geo.kv_pos0;
             if (vlo_ll < 0) vlo_ll = 0;
             if (vhi_ll > geo.kv_len - 1) vhi_ll = geo.kv_len - 1;
             const int vlo = (int)vlo_ll, vhi = (int)vhi_ll;
-            long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.flagged) - geo.kv_pos0;
+            long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.cls) - geo.kv_pos0;
             long long full_hi = (long long)geo.q_pos0 + r0 - geo.kv_pos0;
             if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
             const bool row_ok = r < geo.Lq;
@@ -527,8 +527,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
     const MaskGeom& geo = prm.geom;
     const int c0 = kt * kTile;
     long long rq_lo, rq_hi;
-    const bool flagged = prm.heads.flag[slot] != 0;
-    kv_tile_q_range(geo, c0, flagged, &rq_lo, &rq_hi);
+    const int cls = prm.heads.flag[slot];
+    kv_tile_q_range(geo, c0, cls, &rq_lo, &rq_hi);
     const int qt_lo = (int)(rq_lo / kTile);
     const int n_qt = rq_hi >= rq_lo ? (int)(rq_hi / kTile) - qt_lo + 1 : 0;
     const int n_it = n_qt * prm.g;
@@ -643,7 +643,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
         const int jl = c0 + row;
         const long long jpos = (long long)geo.kv_pos0 + jl;
         // query rows that read this key differentiably: [qlo, qhi]
-        long long qlo_ll = jpos - geo.q_pos0, qhi_ll = hi_diff(geo, jpos < 0 ? 0 : jpos, flagged) - 1 - geo.q_pos0;
+        long long qlo_ll = jpos - geo.q_pos0, qhi_ll = hi_diff(geo, jpos < 0 ? 0 : jpos, cls) - 1 - geo.q_pos0;
         if (jpos < 0) qhi_ll = -1;
         if (qlo_ll < 0) qlo_ll = 0;
         if (qhi_ll > geo.Lq - 1) qhi_ll = geo.Lq - 1;
@@ -651,7 +651,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
         // no element mask when every key row of the tile is read by every query row of the query tile
         const long long jfirst = (long long)geo.kv_pos0 + c0, jlast = jfirst + kTile - 1;
         const long long full_qlo = jlast - geo.q_pos0;  // latest first-reader
-        long long full_qhi = (jfirst >= 0 ? hi_diff(geo, jfirst, flagged) : 0) - 1 - geo.q_pos0;  // earliest last-reader
+        long long full_qhi = (jfirst >= 0 ? hi_diff(geo, jfirst, cls) : 0) - 1 - geo.q_pos0;  // earliest last-reader
         if (full_qhi > geo.Lq - 1) full_qhi = geo.Lq - 1;
         const bool keys_in_range = c0 + kTile <= geo.kv_len && jfirst >= 0;
 

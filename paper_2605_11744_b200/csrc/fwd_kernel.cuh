@@ -43,7 +43,7 @@ struct FwdSmem {
 // visible ranges) before the others, late query tiles before early ones.
 struct FwdItem {
     int b, hq, slot, qt;
-    bool flagged;
+    int cls;  // head class of the item's KV head
 };
 __device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) {
     const HeadTable& ht = prm.heads;
@@ -69,13 +69,13 @@ __device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) {
     it.slot = ht.order[cls_off + t % cls_n];
     it.b = t / cls_n;
     it.hq = ht.logical[it.slot] * prm.g + r;
-    it.flagged = ht.flag[it.slot] != 0;
+    it.cls = ht.flag[it.slot];
     return it;
 }
 // first visible key tile and number of visible key tiles of a work item
 __device__ __forceinline__ void fwd_item_tiles(const FwdParams& prm, const FwdItem& it, int* t_lo, int* n_tiles) {
     long long jl_lo, jl_hi;
-    q_tile_kv_range(prm.geom, it.qt * kTile, it.flagged, false, &jl_lo, &jl_hi);
+    q_tile_kv_range(prm.geom, it.qt * kTile, it.cls, false, &jl_lo, &jl_hi);
     *t_lo = (int)(jl_lo / kTile);
     *n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - *t_lo + 1 : 0;
 }
@@ -292,13 +292,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             const int r = r0 + row;
             const long long p = (long long)geo.q_pos0 + r;
             // visible local key rows of this query row: [vlo, vhi]
-            long long vlo_ll = lo_visible(geo, p, it.flagged) - geo.kv_pos0;
+            long long vlo_ll = lo_visible(geo, p, it.cls) - geo.kv_pos0;
             long long vhi_ll = p - geo.kv_pos0;
             if (vlo_ll < 0) vlo_ll = 0;
             if (vhi_ll > geo.kv_len - 1) vhi_ll = geo.kv_len - 1;
             const int vlo = (int)vlo_ll, vhi = (int)vhi_ll;
             // a key tile [c0, c0+128) needs no element mask when every row of the tile sees all of it
-            long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.flagged) - geo.kv_pos0;
+            long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.cls) - geo.kv_pos0;
             long long full_hi = (long long)geo.q_pos0 + r0 - geo.kv_pos0;
             if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
 

@@ -4,8 +4,9 @@
 // Global positions: query row r is position p = q_pos0 + r, key row jl is position
 // j = kv_pos0 + jl.  With i = p / S and a_i = max(0, i*S - T) (start of the carried tail of
 // the previous segment, Section 3.4 "Local Continuity Channel"; C_0 empty, Section 3.1):
-//   visible(p, j) <=> lo_vis(p) <= j <= p,  lo_vis(p) = flagged ? 0 : a_i   (Appendix C, Eq. "ctx")
-//   diff(p, j)    <=> a_i <= j <= p     (reads whose K/V receive gradient; Definition 3.2)
+//   visible(p, j) <=> lo_vis(p) <= j <= p,  lo_vis(p) = a_i, 0 or i*S by head class   (Appendix C, Eq. "ctx")
+//   diff(p, j)    <=> a_i <= j <= p     (reads whose K/V receive gradient; Definition 3.2); i*S <= j <= p
+//                     for an own-segment-only head
 // For a fixed key j the differentiable queries are also one interval: p in [j, hi_diff(j)),
 // hi_diff(j) = end of j's segment, plus the whole next segment when j lies in the last T
 // positions of its segment.
@@ -34,28 +35,37 @@ __host__ __device__ inline long long tail_start(const MaskGeom& g, long long p) 
     long long a = seg_of(p, g.S) * (long long)g.S - g.T;
     return a < 0 ? 0 : a;
 }
-__host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, bool flagged) {
-    return flagged ? 0 : tail_start(g, p);
+// Head classes (Appendix C, Eq. "ctx"): what a KV head's queries read besides their own segment.
+constexpr int kHeadLocal = 0;  // the carried tail of the previous segment, differentiably
+constexpr int kHeadPast = 1;   // every older position; what lies before the tail start is forward-only
+constexpr int kHeadOwn = 2;    // nothing: a long-range head outside the long-range layers
+// own segment only on the K/V-gradient side?
+__host__ __device__ inline bool diff_own_only(const MaskGeom& g, int cls) {
+    return cls == kHeadOwn || (cls == kHeadPast && g.flagged_tail_sg);
 }
-// one past the last query position that differentiably reads key position j (of a flagged head or not)
-__host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, bool flagged) {
+__host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, int cls) {
+    if (cls == kHeadPast) return 0;
+    return cls == kHeadOwn ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
+}
+// one past the last query position that differentiably reads key position j of a head of class cls
+__host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, int cls) {
     long long seg_end = (seg_of(j, g.S) + 1) * (long long)g.S;
-    if (flagged && g.flagged_tail_sg) return seg_end;
+    if (diff_own_only(g, cls)) return seg_end;
     return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
 }
 // first key position query position p reads differentiably
-__host__ __device__ inline long long lo_diff(const MaskGeom& g, long long p, bool flagged) {
-    return (flagged && g.flagged_tail_sg) ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
+__host__ __device__ inline long long lo_diff(const MaskGeom& g, long long p, int cls) {
+    return diff_own_only(g, cls) ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
 }
 
 // Local key-row range [jl_lo, jl_hi] (inclusive) that the query tile starting at row r0 can see;
 // empty when jl_hi < jl_lo.
-__host__ __device__ inline void q_tile_kv_range(const MaskGeom& g, int r0, bool flagged, bool diff_only,
+__host__ __device__ inline void q_tile_kv_range(const MaskGeom& g, int r0, int cls, bool diff_only,
                                                 long long* jl_lo, long long* jl_hi) {
     int r_last = r0 + kTile - 1;
     if (r_last > g.Lq - 1) r_last = g.Lq - 1;
     long long p0 = (long long)g.q_pos0 + r0, p1 = (long long)g.q_pos0 + r_last;
-    long long lo = diff_only ? tail_start(g, p0) : lo_visible(g, p0, flagged);
+    long long lo = diff_only ? lo_diff(g, p0, cls) : lo_visible(g, p0, cls);
     long long a = lo - g.kv_pos0, b = p1 - g.kv_pos0;
     if (a < 0) a = 0;
     if (b > g.kv_len - 1) b = g.kv_len - 1;
@@ -64,14 +74,14 @@ __host__ __device__ inline void q_tile_kv_range(const MaskGeom& g, int r0, bool 
 }
 // Query-row range [r_lo, r_hi] (inclusive) that differentiably reads some key of the key tile
 // starting at local row c0; empty when r_hi < r_lo.
-__host__ __device__ inline void kv_tile_q_range(const MaskGeom& g, int c0, bool flagged, long long* r_lo, long long* r_hi) {
+__host__ __device__ inline void kv_tile_q_range(const MaskGeom& g, int c0, int cls, long long* r_lo, long long* r_hi) {
     int c_last = c0 + kTile - 1;
     if (c_last > g.kv_len - 1) c_last = g.kv_len - 1;
     long long j0 = (long long)g.kv_pos0 + c0, j1 = (long long)g.kv_pos0 + c_last;
     if (j1 < 0) { *r_lo = 0; *r_hi = -1; return; }
     if (j0 < 0) j0 = 0;
     long long a = j0 - g.q_pos0;              // first query position is the key itself
-    long long b = hi_diff(g, j1, flagged) - 1 - g.q_pos0;  // hi_diff is non-decreasing in j
+    long long b = hi_diff(g, j1, cls) - 1 - g.q_pos0;  // hi_diff is non-decreasing in j
     if (a < 0) a = 0;
     if (b > g.Lq - 1) b = g.Lq - 1;
     *r_lo = a;
@@ -81,10 +91,10 @@ __host__ __device__ inline void kv_tile_q_range(const MaskGeom& g, int c0, bool 
 // Which KV "slot" (head index inside the K/V tensors handed to the kernel) serves which
 // logical KV head, in what launch order, and whether it is flagged.
 struct HeadTable {
-    uint8_t order[kMaxKvHeads];    // slots sorted flagged-first (heaviest work first)
-    uint8_t flag[kMaxKvHeads];     // per slot
+    uint8_t order[kMaxKvHeads];    // slots sorted heaviest work first: past-access, local, own-segment-only
+    uint8_t flag[kMaxKvHeads];     // per slot: head class (kHeadLocal / kHeadPast / kHeadOwn)
     uint8_t logical[kMaxKvHeads];  // per slot: logical KV head (query heads logical*g .. +g-1)
-    int n_slots, n_flagged;
+    int n_slots, n_flagged;        // n_flagged: past-access slots (the first n_flagged entries of order)
 };
 
 // The work items a persistent CTA takes, in order: the list is sorted heaviest first and dealt to the

@@ -114,18 +114,28 @@ segattn_status make_map(CUtensorMap* m, const void* base, int d, int heads, long
     return SEGATTN_OK;
 }
 
+// every entry of the per-KV-head class array is one of SEGATTN_HEAD_LOCAL / _PAST / _OWN
+bool mask_ok(const uint8_t* mask, int Hkv) {
+    if (!mask) return false;
+    for (int c = 0; c < Hkv; ++c)
+        if (mask[c] > SEGATTN_HEAD_OWN) return false;
+    return true;
+}
+
 void identity_heads(HeadTable* ht, int Hkv, const uint8_t* mask) {
     ht->n_slots = Hkv;
-    ht->n_flagged = 0;
     int k = 0;
-    for (int c = 0; c < Hkv; ++c) {
-        ht->flag[c] = mask[c] ? 1 : 0;
-        ht->logical[c] = (uint8_t)c;
-        if (mask[c]) ht->order[k++] = (uint8_t)c;
+    // launch order: heaviest class first (past-access, then local, then own-segment-only)
+    const int by_weight[3] = {kHeadPast, kHeadLocal, kHeadOwn};
+    for (int w = 0; w < 3; ++w) {
+        for (int c = 0; c < Hkv; ++c)
+            if (mask[c] == by_weight[w]) ht->order[k++] = (uint8_t)c;
+        if (w == 0) ht->n_flagged = k;
     }
-    ht->n_flagged = k;
-    for (int c = 0; c < Hkv; ++c)
-        if (!mask[c]) ht->order[k++] = (uint8_t)c;
+    for (int c = 0; c < Hkv; ++c) {
+        ht->flag[c] = mask[c];
+        ht->logical[c] = (uint8_t)c;
+    }
 }
 
 MaskGeom geom_of(const seg_attn_params* p) {
@@ -214,7 +224,7 @@ segattn_status seg_attn_fwd(const seg_attn_params* p, const void* Q, const void*
                             size_t workspace_bytes, void* stream) {
     (void)workspace;
     (void)workspace_bytes;
-    if (!params_ok(p) || !head_past_mask) return SEGATTN_ERR_INVALID;
+    if (!params_ok(p) || !mask_ok(head_past_mask, p->Hkv)) return SEGATTN_ERR_INVALID;
     if (!strides_ok(p->q_stride, p->d) || !strides_ok(p->k_stride, p->d) || !strides_ok(p->v_stride, p->d) ||
         !strides_ok(p->o_stride, p->d))
         return SEGATTN_ERR_INVALID;
@@ -264,12 +274,12 @@ int64_t seg_attn_launch_count(void) { return g_launches.load(); }
 
 segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* head_past_mask, int64_t* pairs_visible,
                                     int64_t* pairs_diff, int64_t* fwd_tiles) {
-    if (!params_ok(p) || !head_past_mask) return SEGATTN_ERR_INVALID;
+    if (!params_ok(p) || !mask_ok(head_past_mask, p->Hkv)) return SEGATTN_ERR_INVALID;
     const MaskGeom g = geom_of(p);
     const int grp = p->Hq / p->Hkv;
     long long vis = 0, dif = 0, tiles = 0;
     for (int c = 0; c < p->Hkv; ++c) {
-        const bool f = head_past_mask[c] != 0;
+        const int f = head_past_mask[c];
         long long v = 0, d = 0, t = 0;
         for (int r = 0; r < p->Lq; ++r) {
             const long long pos = (long long)g.q_pos0 + r;
@@ -359,7 +369,7 @@ extern "C" segattn_status seg_attn_bwd_static(const seg_attn_params* p, const vo
                                               const void* O, const float* LSE, const void* dO,
                                               const uint8_t* head_past_mask, void* dQ, void* dK, void* dV,
                                               void* stream) {
-    if (!params_ok(p) || !head_past_mask || !all_strides_ok(p)) return SEGATTN_ERR_INVALID;
+    if (!params_ok(p) || !mask_ok(head_past_mask, p->Hkv) || !all_strides_ok(p)) return SEGATTN_ERR_INVALID;
     const bool have_q = p->B > 0 && p->Lq > 0, have_kv = p->B > 0 && p->kv_len > 0;
     if (have_q && (!Q || !O || !LSE || !dO || !dQ || !aligned16(Q) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
                    (reinterpret_cast<uintptr_t>(LSE) & 3u)))

@@ -100,6 +100,8 @@ def test_no_device_means_an_error_not_a_fallback():
     (2, 1000, 4, 2, 200, 72, [1, 0]),
     (1, 777, 2, 2, 64, 64, [0, 1]),
     (1, 300, 2, 1, 7, 0, [0]),
+    (2, 1000, 4, 2, 200, 72, [2, 1]),       # an own-segment-only head beside a past-access one
+    (1, 777, 3, 3, 64, 64, [2, 0, 1]),      # all three head classes
 ])
 def test_pair_counter_matches_oracle_enumeration(B, L, Hq, Hkv, S, T, mask):
     nv, nd, tiles = sa.count_pairs(B, L, Hq, Hkv, 128, S, T, mask)
@@ -109,6 +111,11 @@ def test_pair_counter_matches_oracle_enumeration(B, L, Hq, Hkv, S, T, mask):
     nv2, nd2, _ = sa.count_pairs(B, L, Hq, Hkv, 128, S, T, mask, flagged_tail_is_sg=True)
     assert (nv2, nd2) == oracle.count_pairs(B, L, Hq, Hkv, S, T, mask, flagged_tail_is_sg=True)
     assert nv2 == nv and nd2 <= nd
+
+
+def test_unknown_head_class_is_rejected():
+    with pytest.raises(sa.SegAttnError):
+        sa.count_pairs(1, 256, 2, 2, 128, 64, 16, [0, 3])
 
 
 def test_benchmark_configuration_counts():

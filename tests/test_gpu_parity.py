@@ -41,6 +41,32 @@ def test_small_cases_match_oracle_elementwise(B, L, Hq, Hkv, d, S, T, mask):
 
 
 @pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask", [
+    (1, 1024, 4, 2, 128, 256, 128, [2, 0]),           # own-segment-only beside local
+    (2, 700, 6, 3, 128, 200, 72, [1, 2, 0]),          # all three classes, nothing aligned, ragged end
+    (1, 1152, 4, 4, 128, 384, 128, [2, 2, 1, 0]),     # segments of three tiles
+    (1, 333, 2, 2, 64, 100, 100, [2, 2]),             # d = 64, every head own-only
+    (1, 640, 2, 2, 128, 64, 64, [2, 1]),              # segments shorter than a tile
+])
+@pytest.mark.parametrize("tail_sg", [False, True])
+def test_head_classes_local_past_and_own_segment_only(B, L, Hq, Hkv, d, S, T, mask, tail_sg):
+    # the three contexts of Eq. "ctx": [tail ; own], [past ; own] and own alone, chosen per KV head
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=L + S + T)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask, flagged_tail_is_sg=tail_sg)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, mask)
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask, flagged_tail_is_sg=tail_sg)
+    assert_fwd_close(O, LSE, Oo, LSEo, "fwd")
+    assert_grads_close((dQ, dK, dV), ref, "bwd")
+    # an own-segment-only head never reads the tail: T does not matter for it, to the bit
+    O0, LSE0 = sa.seg_attn_fwd(Q, K, V, S, 0, mask)
+    g = Hq // Hkv
+    for c, cls in enumerate(mask):
+        if cls == 2:
+            assert torch.equal(O[:, :, c * g:(c + 1) * g], O0[:, :, c * g:(c + 1) * g])
+
+
+@pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask", [
     (1, 1024, 4, 2, 128, 256, 128, [0, 1]),
     (2, 700, 4, 2, 128, 200, 72, [1, 0]),
     (1, 640, 2, 2, 128, 64, 64, [1, 1]),
@@ -59,7 +85,7 @@ def test_flagged_heads_reading_the_tail_forward_only(B, L, Hq, Hkv, d, S, T, mas
     assert torch.equal(dQ, dQ0)
     for c, f in enumerate(mask):
         same = torch.equal(dK[:, :, c], dK0[:, :, c]) and torch.equal(dV[:, :, c], dV0[:, :, c])
-        assert same == (not f or T == 0)
+        assert same == (f != 1 or T == 0)
 
 
 def test_window_of_queries_with_position_offsets():

@@ -35,6 +35,7 @@ def run_streamed(Q, K, V, S, T, mask, scale=None):
     (1, 800, 2, 2, 64, 200, 72, [0, 1]),        # tiles of the window do not line up with the one-shot tiles
     (1, 512, 2, 2, 128, 128, 128, [0, 0]),
     (1, 512, 2, 1, 128, 128, 64, [1]),
+    (1, 1024, 4, 4, 128, 256, 128, [2, 1, 0, 2]),   # all three head classes; own-only heads ignore the window's tail
 ])
 def test_streamed_equals_one_shot_and_oracle(B, L, Hq, Hkv, d, S, T, mask):
     Q, K, V, _ = rand_inputs(B, L, Hq, Hkv, d, seed=L + T)
