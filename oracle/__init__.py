@@ -27,7 +27,7 @@ _lib = None
 
 class _Cfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
-                ("B", "Lq", "Lk", "Hq", "Hkv", "d", "S", "T", "q_pos0", "kv_pos0", "flagged_tail_is_sg")] + \
+                ("B", "Lq", "Lk", "Hq", "Hkv", "d", "S", "T", "q_pos0", "kv_pos0", "flagged_tail_is_sg", "detach_before")] + \
                [("scale", ctypes.c_double)]
 
 
@@ -64,13 +64,13 @@ def _ptr(a):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
 
 
-def _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg):
+def _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg, detach_before=0):
     B, Lq, Hq, d = Q.shape
     Bk, Lk, Hkv, dk = K.shape
     assert B == Bk and d == dk and Hq % Hkv == 0
     if scale is None:
         scale = 1.0 / np.sqrt(d)
-    return _Cfg(B, Lq, Lk, Hq, Hkv, d, S, T, q_pos0, kv_pos0, int(bool(flagged_tail_is_sg)), float(scale))
+    return _Cfg(B, Lq, Lk, Hq, Hkv, d, S, T, q_pos0, kv_pos0, int(bool(flagged_tail_is_sg)), int(detach_before), float(scale))
 
 
 def _mask(head_past_mask, Hkv):
@@ -94,10 +94,12 @@ def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, fla
     return O, LSE
 
 
-def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False):
-    """dQ, dK, dV for the cotangent dO; dK/dV hold only what the queries passed in contribute."""
+def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False,
+        detach_before=0):
+    """dQ, dK, dV for the cotangent dO; dK/dV hold only what the queries passed in contribute.  Keys at
+    global positions below ``detach_before`` are read forward-only (a window with a detached incoming state)."""
     Q, K, V, dO = _f64(Q), _f64(K), _f64(V), _f64(dO)
-    cfg = _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg)
+    cfg = _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg, detach_before)
     m = _mask(head_past_mask, cfg.Hkv)
     dQ, dK, dV = np.empty_like(Q), np.empty_like(K), np.empty_like(V)
     rc = _load().oracle_seg_attn_bwd(ctypes.byref(cfg), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO),
@@ -108,9 +110,9 @@ def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0,
     return dQ, dK, dV
 
 
-def count_pairs(B, L, Hq, Hkv, S, T, head_past_mask=None, flagged_tail_is_sg=False):
+def count_pairs(B, L, Hq, Hkv, S, T, head_past_mask=None, flagged_tail_is_sg=False, detach_before=0):
     """(visible, differentiable) query-key pair counts by enumerating the mask row by row."""
-    cfg = _Cfg(B, L, L, Hq, Hkv, 1, S, T, 0, 0, int(bool(flagged_tail_is_sg)), 1.0)
+    cfg = _Cfg(B, L, L, Hq, Hkv, 1, S, T, 0, 0, int(bool(flagged_tail_is_sg)), int(detach_before), 1.0)
     m = _mask(head_past_mask, Hkv)
     nv, nd = ctypes.c_int64(), ctypes.c_int64()
     rc = _load().oracle_count_pairs(ctypes.byref(cfg), m.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)),

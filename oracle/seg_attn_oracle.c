@@ -23,6 +23,12 @@
  *     start, dense (no top-k retrieval), in union with the tail and the own
  *     segment.  With flagged_tail_is_sg != 0 the flagged head's tail reads are
  *     stop-gradient too (the variant where only local heads carry the state).
+ *   - detach_before: in the K-truncated objective the state at the truncation
+ *     boundary enters as a constant, sg(C_b) (definition of the K-truncated
+ *     consistent objective, Eq. "truncated-base").  A call on a window of
+ *     segments passes the global position where its differentiable part starts;
+ *     every read of a key before it is stop-gradient: diff additionally
+ *     requires j >= detach_before.  0 leaves the mask as stated.
  *   - head_past_mask[c] is a head class: 0 local, 1 flagged as above, 2 a head
  *     whose context is its own segment alone (the long-range head of a layer
  *     outside the long-range layers, Appendix C, Eq. "ctx", third case):
@@ -59,6 +65,7 @@ typedef struct {
     int32_t S, T;
     int32_t q_pos0, kv_pos0;
     int32_t flagged_tail_is_sg;
+    int32_t detach_before;   /* keys at global positions below this are read forward-only; 0: none */
     double scale;
 } oracle_cfg;
 
@@ -67,7 +74,7 @@ static int cfg_ok(const oracle_cfg *c)
     if (c->B < 0 || c->Lq < 0 || c->Lk < 0 || c->Hq <= 0 || c->Hkv <= 0 || c->d <= 0) return 0;
     if (c->Hq % c->Hkv) return 0;
     if (c->S <= 0 || c->T < 0 || c->T > c->S) return 0;
-    if (c->q_pos0 < 0) return 0;
+    if (c->q_pos0 < 0 || c->detach_before < 0) return 0;
     return 1;
 }
 
@@ -79,10 +86,13 @@ static void row_bounds(const oracle_cfg *c, int flag, long p, long *lo_vis, long
     if (a < 0) a = 0;
     if (flag == 2) {             /* own segment only (Appendix C, Eq. "ctx", third case) */
         *lo_vis = *lo_diff = i * (long)c->S;
-        return;
+    } else {
+        *lo_vis = flag ? 0 : a;
+        *lo_diff = (flag && c->flagged_tail_is_sg) ? i * (long)c->S : a;
     }
-    *lo_vis = flag ? 0 : a;
-    *lo_diff = (flag && c->flagged_tail_is_sg) ? i * (long)c->S : a;
+    /* the boundary state of a truncated chain is a constant (Eq. "truncated-base"): reads of keys
+     * before detach_before carry no gradient into K/V */
+    if (*lo_diff < c->detach_before) *lo_diff = c->detach_before;
 }
 
 /* One query row: scores, LSE, probabilities P[jl] for jl in [j0,j1) (local key

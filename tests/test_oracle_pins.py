@@ -105,11 +105,15 @@ def test_own_segment_only_heads_are_block_diagonal_for_any_tail():
     np.testing.assert_allclose(dense.fwd(Q, K, V, S, T, head_past_mask=[2, 0])[0], O, atol=TOL)
 
 
-def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False):
+def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False, detach_before=0):
     """For every segment i and head: context = [sg(older past) if flagged ; tail of segment i-1 ;
     own segment], every prefix position visible and the own segment causal (Appendix C), run
     through library attention; stop-gradient realised with .detach() (Definition 3.2)."""
-    q, k, v = t64(Q, True), t64(K, True), t64(V, True)
+    q, k0, v0 = t64(Q, True), t64(K, True), t64(V, True)
+    # keys before detach_before enter as constants (the boundary state of a truncated chain)
+    X = detach_before
+    k = torch.cat([k0[:, :X].detach(), k0[:, X:]], dim=1)
+    v = torch.cat([v0[:, :X].detach(), v0[:, X:]], dim=1)
     B, L, Hq, d = Q.shape
     Hkv = K.shape[2]
     g = Hq // Hkv
@@ -144,7 +148,7 @@ def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False):
             sc = torch.einsum("bld,bmd->blm", q[:, s0:s1, h], kc) / np.sqrt(d)
             lses[:, h, s0:s1] = torch.logsumexp(sc.masked_fill(~m, float("-inf")), dim=-1).detach()
     torch.stack(pieces).sum().backward()
-    return outs.numpy(), lses.numpy(), q.grad.numpy(), k.grad.numpy(), v.grad.numpy()
+    return outs.numpy(), lses.numpy(), q.grad.numpy(), k0.grad.numpy(), v0.grad.numpy()
 
 
 @pytest.mark.parametrize("L,S,T,flags,variant", [
@@ -172,6 +176,45 @@ def test_segment_recurrence_with_autograd(L, S, T, flags, variant):
         d2 = dense.bwd(Q, K, V, dO, S, T, head_past_mask=flags)
         for a, b in zip((dQ, dK, dV), d2):
             np.testing.assert_allclose(a, b, atol=TOL)
+
+
+@pytest.mark.parametrize("L,S,T,flags,X", [
+    (96, 32, 8, [0, 1], 32),      # the window's differentiable part starts at segment 1
+    (96, 32, 8, [0, 1], 64),
+    (100, 32, 32, [2, 0], 40),    # a boundary inside a segment, ragged end
+    (96, 32, 8, [1, 1], 96),      # everything detached: no K/V gradient at all
+])
+def test_detached_prefix_equals_autograd_with_constant_keys(L, S, T, flags, X):
+    Q, K, V, dO = rand(2, L, 4, 2, 8)
+    o, lse, gq, gk, gv = recurrence_autograd(Q, K, V, dO, S, T, flags, detach_before=X)
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, T, head_past_mask=flags, detach_before=X)
+    np.testing.assert_allclose(dQ, gq, atol=TOL)
+    np.testing.assert_allclose(dK, gk, atol=TOL)
+    np.testing.assert_allclose(dV, gv, atol=TOL)
+    assert not dK[:, :X].any() and not dV[:, :X].any()
+    # dQ does not depend on where K/V are cut
+    np.testing.assert_array_equal(dQ, oracle.bwd(Q, K, V, dO, S, T, head_past_mask=flags)[0])
+
+
+def test_windows_with_detached_incoming_state_compose_to_depth_one_truncation():
+    # Truncation depth 1 over one layer: the loss of segment i sends gradient into the K/V of segments
+    # i-1 (its tail) and i only.  Summing, over windows [i-1, i] whose incoming state is detached, the
+    # gradients of the window's LAST segment loss gives the gradient of the whole untruncated call,
+    # because one attention layer has no longer state chain than one transition.
+    L, S, T = 128, 32, 8
+    Q, K, V, dO = rand(1, L, 2, 2, 8)
+    full = oracle.bwd(Q, K, V, dO, S, T)
+    acc = [np.zeros_like(a) for a in full]
+    for i in range(L // S):
+        lo = max(0, i - 1) * S
+        sl = slice(lo, (i + 1) * S)
+        dOw = dO[:, sl].copy()
+        dOw[:, :i * S - lo] = 0.0                      # only segment i's loss term
+        g = oracle.bwd(Q[:, sl], K[:, sl], V[:, sl], dOw, S, T, q_pos0=lo, kv_pos0=lo, detach_before=lo)
+        for a, b in zip(acc, g):
+            a[:, sl] += b
+    for a, b in zip(acc, full):
+        np.testing.assert_allclose(a, b, atol=TOL)
 
 
 # ---- closed form: zero keys => uniform attention over the visible set ---------------------------
