@@ -85,6 +85,11 @@ typedef struct {
     int32_t kv_pos0; /* global position of key row 0 (may be negative: rows before position 0 are never visible) */
     float sm_scale;  /* softmax scale; the paper uses 1/sqrt(d) */
     int32_t flags;   /* bit set of SEGATTN_FLAG_*; 0 for the default semantics */
+    int32_t detach_before; /* backward only: keys at global positions below this are read forward-only
+                            * (no dK/dV from them, and their dK/dV rows come out zero): the boundary
+                            * state of a truncated chain enters as a constant (K-truncated objective,
+                            * Eq. "truncated-base").  A window of K+1 segments passes the position of
+                            * its first segment.  0: none.  Must be >= 0. */
     int64_t q_stride[3]; /* element strides of Q (and dQ) for (batch, position, head) */
     int64_t k_stride[3]; /* element strides of K (and dK) */
     int64_t v_stride[3]; /* element strides of V (and dV) */

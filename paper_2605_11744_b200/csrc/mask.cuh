@@ -23,6 +23,7 @@ struct MaskGeom {
     int S, T;
     int q_pos0, kv_pos0;
     int Lq, kv_len;
+    int detach_before;    // keys before this global position are read forward-only (0: none)
     int flagged_tail_sg;  // flagged heads read the carried tail forward-only too (Appendix C, Eq. "ctx", read literally)
 };
 
@@ -49,13 +50,15 @@ __host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, 
 }
 // one past the last query position that differentiably reads key position j of a head of class cls
 __host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, int cls) {
+    if (j < g.detach_before) return j;  // no differentiable reader at all
     long long seg_end = (seg_of(j, g.S) + 1) * (long long)g.S;
     if (diff_own_only(g, cls)) return seg_end;
     return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
 }
 // first key position query position p reads differentiably
 __host__ __device__ inline long long lo_diff(const MaskGeom& g, long long p, int cls) {
-    return diff_own_only(g, cls) ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
+    const long long lo = diff_own_only(g, cls) ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
+    return lo < g.detach_before ? g.detach_before : lo;
 }
 
 // Local key-row range [jl_lo, jl_hi] (inclusive) that the query tile starting at row r0 can see;
@@ -80,6 +83,8 @@ __host__ __device__ inline void kv_tile_q_range(const MaskGeom& g, int c0, int c
     long long j0 = (long long)g.kv_pos0 + c0, j1 = (long long)g.kv_pos0 + c_last;
     if (j1 < 0) { *r_lo = 0; *r_hi = -1; return; }
     if (j0 < 0) j0 = 0;
+    if (j0 < g.detach_before) j0 = g.detach_before;  // keys before it have no differentiable reader
+    if (j0 > j1) { *r_lo = 0; *r_hi = -1; return; }
     long long a = j0 - g.q_pos0;              // first query position is the key itself
     long long b = hi_diff(g, j1, cls) - 1 - g.q_pos0;  // hi_diff is non-decreasing in j
     if (a < 0) a = 0;

@@ -80,7 +80,7 @@ bool params_ok(const seg_attn_params* p) {
     if (p->Hq <= 0 || p->Hkv <= 0 || p->Hkv > kMaxKvHeads || p->Hq % p->Hkv) return false;
     if (p->d != 64 && p->d != 128) return false;
     if (p->S < 1 || p->T < 0 || p->T > p->S) return false;
-    if (p->q_pos0 < 0) return false;
+    if (p->q_pos0 < 0 || p->detach_before < 0) return false;
     if (p->flags & ~SEGATTN_FLAG_FLAGGED_TAIL_SG) return false;
     if (!(p->sm_scale > 0.f) || !std::isfinite(p->sm_scale)) return false;
     if ((long long)p->q_pos0 + p->Lq > 0x7fffffffLL / 2) return false;
@@ -147,6 +147,7 @@ MaskGeom geom_of(const seg_attn_params* p) {
     g.Lq = p->Lq;
     g.kv_len = p->kv_len;
     g.flagged_tail_sg = (p->flags & SEGATTN_FLAG_FLAGGED_TAIL_SG) ? 1 : 0;
+    g.detach_before = p->detach_before;
     return g;
 }
 

@@ -113,6 +113,14 @@ def test_pair_counter_matches_oracle_enumeration(B, L, Hq, Hkv, S, T, mask):
     assert nv2 == nv and nd2 <= nd
 
 
+def test_pair_counter_with_a_detached_prefix():
+    for X in (0, 200, 300, 1000):
+        nv, nd, _ = sa.count_pairs(2, 1000, 4, 2, 128, 200, 72, [1, 0], detach_before=X)
+        assert (nv, nd) == oracle.count_pairs(2, 1000, 4, 2, 200, 72, [1, 0], detach_before=X)
+    with pytest.raises(sa.SegAttnError):
+        sa.count_pairs(1, 256, 2, 2, 128, 64, 16, [0, 0], detach_before=-1)
+
+
 def test_unknown_head_class_is_rejected():
     with pytest.raises(sa.SegAttnError):
         sa.count_pairs(1, 256, 2, 2, 128, 64, 16, [0, 3])

@@ -66,6 +66,42 @@ def test_head_classes_local_past_and_own_segment_only(B, L, Hq, Hkv, d, S, T, ma
             assert torch.equal(O[:, :, c * g:(c + 1) * g], O0[:, :, c * g:(c + 1) * g])
 
 
+@pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask,X", [
+    (1, 1024, 4, 2, 128, 256, 128, [0, 1], 256),      # boundary on a segment and a tile
+    (2, 700, 4, 2, 128, 200, 72, [1, 0], 400),        # boundary inside a tile
+    (1, 1152, 6, 3, 128, 384, 128, [2, 1, 0], 500),   # boundary inside a segment, all head classes
+    (1, 333, 2, 2, 64, 100, 100, [0, 1], 333),        # everything detached
+    (1, 640, 2, 1, 128, 128, 64, [0], 0),             # none
+])
+def test_detached_prefix_gets_no_gradient(B, L, Hq, Hkv, d, S, T, mask, X):
+    # keys before detach_before are constants of the window (the boundary state of a truncated chain)
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=L + X)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask, detach_before=X)
+    sa.poll_status()
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask, detach_before=X)
+    assert_grads_close((dQ, dK, dV), ref, "detached prefix")
+    assert not dK[:, :X].any() and not dV[:, :X].any()
+    dQ0, _, _ = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask)
+    assert torch.equal(dQ, dQ0)
+
+
+def test_window_of_two_segments_with_detached_incoming_tail():
+    # one step of depth-one truncation: queries of segments i-1 and i, keys from the tail of segment i-2 on;
+    # that tail is read (forward) but receives nothing
+    B, L, Hq, Hkv, d, S, T = 1, 1024, 4, 2, 128, 256, 128
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=5)
+    lo, k0 = 2 * S, 2 * S - T
+    Qw, dOw = Q[:, lo:lo + 2 * S].contiguous(), dO[:, lo:lo + 2 * S].contiguous()
+    Kw, Vw = K[:, k0:lo + 2 * S].contiguous(), V[:, k0:lo + 2 * S].contiguous()
+    Ow, LSEw = sa.seg_attn_fwd(Qw, Kw, Vw, S, T, [0, 0], q_pos0=lo, kv_pos0=k0)
+    g = sa.seg_attn_bwd(Qw, Kw, Vw, Ow, LSEw, dOw, S, T, [0, 0], q_pos0=lo, kv_pos0=k0, detach_before=lo)
+    sa.poll_status()
+    ref = oracle.bwd(f64(Qw), f64(Kw), f64(Vw), f64(dOw), S, T, [0, 0], q_pos0=lo, kv_pos0=k0, detach_before=lo)
+    assert_grads_close(g, ref, "window")
+    assert not g[1][:, :T].any() and not g[2][:, :T].any()
+
+
 @pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask", [
     (1, 1024, 4, 2, 128, 256, 128, [0, 1]),
     (2, 700, 4, 2, 128, 200, 72, [1, 0]),
