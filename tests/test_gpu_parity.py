@@ -308,6 +308,23 @@ def test_host_buffer_step_matches_device_path():
         assert torch.equal(outs[k], t.cpu()), k
 
 
+@pytest.mark.parametrize("B", [2, 6])
+def test_host_buffer_step_in_overlapped_chunks(B):
+    # the host-buffer step cuts the batch into chunks (here of unequal size for B = 6) whose copies and
+    # kernels overlap on separate streams: the results are those of one launch over the whole batch
+    L, Hq, Hkv, d, S, T, mask = 640, 4, 2, 128, 256, 128, [1, 0]
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=B, device="cpu")
+    for forward_only in (False, True):
+        outs = sa.seg_attn_step_host(Q, K, V, None if forward_only else dO, S, T, mask)
+        Qd, Kd, Vd, dOd = (t.cuda() for t in (Q, K, V, dO))
+        O, LSE = sa.seg_attn_fwd(Qd, Kd, Vd, S, T, mask)
+        assert torch.equal(outs["O"], O.cpu()) and torch.equal(outs["LSE"], LSE.cpu())
+        if not forward_only:
+            dQ, dK, dV = sa.seg_attn_bwd(Qd, Kd, Vd, O, LSE, dOd, S, T, mask)
+            for k, t in (("dQ", dQ), ("dK", dK), ("dV", dV)):
+                assert torch.equal(outs[k], t.cpu()), k
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
     # a wait on a barrier nothing signals gives up after its limit and sets the status word: no hang, no fault
     sa.poll_status()
