@@ -37,9 +37,9 @@ UNIT = "TFLOP/s"
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on the
 # benchmark workload, taken from the ncu captures summarised under profiles/; None = not captured.
 NCU_TRAFFIC_BYTES = {
-    ("cfg2_gqa16k", "fwd"): 651273216,
-    ("cfg2_gqa16k", "dq"): 938126848,
-    ("cfg2_gqa16k", "dkv"): 804103424,
+    ("cfg2_gqa16k", "fwd"): 647472896,
+    ("cfg2_gqa16k", "dq"): 931462912,
+    ("cfg2_gqa16k", "dkv"): 799191552,
 }
 
 
