@@ -238,6 +238,40 @@ def test_empty_and_degenerate_shapes():
     assert torch.count_nonzero(dQ[:, 128:]) == 0
 
 
+def test_limits_of_the_interface():
+    # 64 KV heads (the most the head table holds), all three classes, one query head each
+    Hkv = 64
+    mask = [(c * 7) % 3 for c in range(Hkv)]
+    Q, K, V, dO = rand_inputs(1, 300, Hkv, Hkv, 64, seed=64)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, 100, 40, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, 100, 40, mask)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), 100, 40, mask)
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), 100, 40, mask)
+    assert_fwd_close(O, LSE, Oo, LSEo, "64 KV heads")
+    assert_grads_close((dQ, dK, dV), ref, "64 KV heads")
+    with pytest.raises(sa.SegAttnError):
+        sa.seg_attn_fwd(*rand_inputs(1, 128, 65, 65, 64, seed=1)[:3], 64, 0, [0] * 65)
+    # positions near the top of the supported range (q_pos0 + Lq <= 2^30 - 1): the segment arithmetic
+    # must not wrap; keys start one tail before the window
+    S, T, L = 4096, 512, 512
+    q0 = (1 << 30) - 1 - L
+    q0 -= q0 % 128
+    k0 = q0 - (q0 % S) - T          # from the tail of the previous segment on
+    Lk = q0 + L - k0
+    Q, K, V, dO = rand_inputs(1, L, 2, 2, 128, seed=30, Lk=Lk)
+    mask = [0, 2]
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask, q_pos0=q0, kv_pos0=k0)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask, q_pos0=q0, kv_pos0=k0)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, mask, q_pos0=q0, kv_pos0=k0)
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask, q_pos0=q0, kv_pos0=k0)
+    assert_fwd_close(O, LSE, Oo, LSEo, "high positions")
+    assert_grads_close((dQ, dK, dV), ref, "high positions")
+    with pytest.raises(sa.SegAttnError):
+        sa.seg_attn_fwd(Q, K, V, S, T, mask, q_pos0=(1 << 30), kv_pos0=k0)
+
+
 def test_invalid_arguments_are_rejected_before_launch():
     Q, K, V, dO = rand_inputs(1, 128, 2, 1, 128)
     with pytest.raises(sa.SegAttnError) as e:
