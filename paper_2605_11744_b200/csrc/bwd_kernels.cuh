@@ -102,24 +102,30 @@ __device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) {
     const int per_u = (ht.n_slots - ht.n_flagged) * prm.g * prm.B;
     const int n_f = per_f * prm.n_qtiles;
     DqItem it;
-    int hb, cls_off, cls_n;
+    // quotient and remainder through the launch-time reciprocals (the operands are small and non-negative)
+    uint32_t q, hb, cls_off, cls_n;
+    FastDiv f_cls;
     if (idx < n_f) {
-        it.qt = prm.n_qtiles - 1 - idx / per_f;
-        hb = idx % per_f;
+        q = fdiv((uint32_t)idx, prm.f_per_f);
+        hb = (uint32_t)idx - q * (uint32_t)per_f;
         cls_off = 0;
-        cls_n = ht.n_flagged;
+        cls_n = (uint32_t)ht.n_flagged;
+        f_cls = prm.f_ncls_f;
     } else {
         idx -= n_f;
-        it.qt = prm.n_qtiles - 1 - idx / per_u;
-        hb = idx % per_u;
-        cls_off = ht.n_flagged;
-        cls_n = ht.n_slots - ht.n_flagged;
+        q = fdiv((uint32_t)idx, prm.f_per_u);
+        hb = (uint32_t)idx - q * (uint32_t)per_u;
+        cls_off = (uint32_t)ht.n_flagged;
+        cls_n = (uint32_t)(ht.n_slots - ht.n_flagged);
+        f_cls = prm.f_ncls_u;
     }
-    const int r = hb % prm.g;
-    const int t = hb / prm.g;
-    it.slot = ht.order[cls_off + t % cls_n];
-    it.b = t / cls_n;
-    it.hq = ht.logical[it.slot] * prm.g + r;
+    it.qt = prm.n_qtiles - 1 - (int)q;
+    const uint32_t t = fdiv(hb, prm.f_g);
+    const uint32_t r = hb - t * (uint32_t)prm.g;
+    const uint32_t bb = fdiv(t, f_cls);
+    it.slot = ht.order[cls_off + (t - bb * cls_n)];
+    it.b = (int)bb;
+    it.hq = ht.logical[it.slot] * prm.g + (int)r;
     it.cls = ht.flag[it.slot];
     return it;
 }

@@ -19,7 +19,33 @@ namespace segattn {
 constexpr int kTile = 128;     // query rows per tile = key rows per tile
 constexpr int kMaxKvHeads = 64;
 
+// Division of a 32-bit unsigned number by a divisor fixed at launch: q = (mulhi(n, m) + n) >> s with
+// s = ceil(log2 d), m = floor(2^32 (2^s - d) / d) + 1 (exact for every 32-bit n).  The device's own
+// 32-bit division is tens of dependent instructions, and a work item's decode needs several.
+struct FastDiv {
+    uint32_t d, m, s;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f;
+    if (d == 0) d = 1;  // never used as a divisor then; keeps the fields defined
+    uint32_t s = 0;
+    while (s < 32 && (1ull << s) < d) ++s;
+    f.d = d;
+    f.s = s;
+    f.m = (uint32_t)((((1ull << s) - d) << 32) / d + 1);
+    return f;
+}
+__host__ __device__ inline uint32_t fdiv(uint32_t n, const FastDiv& f) {
+#ifdef __CUDA_ARCH__
+    const uint32_t hi = __umulhi(n, f.m);
+#else
+    const uint32_t hi = (uint32_t)(((unsigned long long)n * f.m) >> 32);
+#endif
+    return (uint32_t)(((unsigned long long)hi + n) >> f.s);
+}
+
 struct MaskGeom {
+    FastDiv fS;  // division by S
     int S, T;
     int q_pos0, kv_pos0;
     int Lq, kv_len;
@@ -27,13 +53,12 @@ struct MaskGeom {
     int flagged_tail_sg;  // flagged heads read the carried tail forward-only too (Appendix C, Eq. "ctx", read literally)
 };
 
-// p / S for a non-negative position: positions fit 32 bits in practice, and a 32-bit division is
-// several times cheaper on the device than a 64-bit one (these run per work item in every thread)
-__host__ __device__ inline long long seg_of(long long p, int S) {
-    return p <= 0xffffffffLL ? (long long)((unsigned)p / (unsigned)S) : p / S;
+// p / S for a non-negative position (positions fit 32 bits: q_pos0 + Lq is limited to 2^30)
+__host__ __device__ inline long long seg_of(const MaskGeom& g, long long p) {
+    return p <= 0xffffffffLL ? (long long)fdiv((uint32_t)p, g.fS) : p / g.S;
 }
 __host__ __device__ inline long long tail_start(const MaskGeom& g, long long p) {
-    long long a = seg_of(p, g.S) * (long long)g.S - g.T;
+    long long a = seg_of(g, p) * (long long)g.S - g.T;
     return a < 0 ? 0 : a;
 }
 // Head classes (Appendix C, Eq. "ctx"): what a KV head's queries read besides their own segment.
@@ -46,18 +71,18 @@ __host__ __device__ inline bool diff_own_only(const MaskGeom& g, int cls) {
 }
 __host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, int cls) {
     if (cls == kHeadPast) return 0;
-    return cls == kHeadOwn ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
+    return cls == kHeadOwn ? seg_of(g, p) * (long long)g.S : tail_start(g, p);
 }
 // one past the last query position that differentiably reads key position j of a head of class cls
 __host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, int cls) {
     if (j < g.detach_before) return j;  // no differentiable reader at all
-    long long seg_end = (seg_of(j, g.S) + 1) * (long long)g.S;
+    long long seg_end = (seg_of(g, j) + 1) * (long long)g.S;
     if (diff_own_only(g, cls)) return seg_end;
     return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
 }
 // first key position query position p reads differentiably
 __host__ __device__ inline long long lo_diff(const MaskGeom& g, long long p, int cls) {
-    const long long lo = diff_own_only(g, cls) ? seg_of(p, g.S) * (long long)g.S : tail_start(g, p);
+    const long long lo = diff_own_only(g, cls) ? seg_of(g, p) * (long long)g.S : tail_start(g, p);
     return lo < g.detach_before ? g.detach_before : lo;
 }
 
@@ -131,6 +156,7 @@ struct alignas(64) FwdParams {
     int B, Hq, g;
     int n_qtiles;
     int n_items;       // work items: B * query heads served * n_qtiles
+    FastDiv f_per_f, f_per_u, f_g, f_ncls_f, f_ncls_u;  // divisors of the work-list decode (see fwd_decode)
     float scale_log2;  // sm_scale * log2(e)
     HeadTable heads;
 };
@@ -148,6 +174,7 @@ struct alignas(64) BwdParams {
     int B, Hq, Hkv, g;
     int n_qtiles, n_kvtiles;
     int n_items_dq;    // work items of the dQ pass: B * query heads served * n_qtiles
+    FastDiv f_per_f, f_per_u, f_g, f_ncls_f, f_ncls_u;  // divisors of the work-list decode (see dq_decode)
     int dkv_tps, dkv_tail_tiles, dkv_n_seg;  // dK/dV grid: key tiles per segment, of which in the tail, segments
     float scale_log2;  // sm_scale * log2(e)
     float sm_scale;

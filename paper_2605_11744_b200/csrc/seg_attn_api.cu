@@ -138,8 +138,19 @@ void identity_heads(HeadTable* ht, int Hkv, const uint8_t* mask) {
     }
 }
 
+// launch-time reciprocals of the work-list decode (fwd_decode / dq_decode)
+template <class Params>
+void set_decode_divisors(Params& prm, const HeadTable& ht, int g, int B) {
+    prm.f_per_f = make_fastdiv((uint32_t)(ht.n_flagged * g * B));
+    prm.f_per_u = make_fastdiv((uint32_t)((ht.n_slots - ht.n_flagged) * g * B));
+    prm.f_g = make_fastdiv((uint32_t)g);
+    prm.f_ncls_f = make_fastdiv((uint32_t)ht.n_flagged);
+    prm.f_ncls_u = make_fastdiv((uint32_t)(ht.n_slots - ht.n_flagged));
+}
+
 MaskGeom geom_of(const seg_attn_params* p) {
     MaskGeom g;
+    g.fS = make_fastdiv((uint32_t)p->S);
     g.S = p->S;
     g.T = p->T;
     g.q_pos0 = p->q_pos0;
@@ -194,6 +205,7 @@ segattn_status launch_fwd(const seg_attn_params* p, const HeadTable& heads, cons
     const long long n_items = (long long)p->B * heads.n_slots * prm.g * prm.n_qtiles;
     if (n_items > 0x7fffffffLL) return SEGATTN_ERR_INVALID;
     prm.n_items = (int)n_items;
+    set_decode_divisors(prm, heads, prm.g, p->B);
     // persistent: one CTA per SM walks the work list
     int n_sm = 0;
     if ((st = sm_count(&n_sm)) != SEGATTN_OK) return st;

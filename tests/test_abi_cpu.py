@@ -121,6 +121,25 @@ def test_pair_counter_with_a_detached_prefix():
         sa.count_pairs(1, 256, 2, 2, 128, 64, 16, [0, 0], detach_before=-1)
 
 
+@pytest.mark.parametrize("S", [1, 2, 3, 7, 100, 127, 128, 1000, 4096, 12345, 65537])
+def test_segment_arithmetic_for_many_segment_lengths(S):
+    # the library divides positions by S through a launch-time reciprocal: check it against the oracle's
+    # plain division, at low positions and near the top of the supported range
+    T = min(S, 5)
+    for L in (1, 257, 3000):
+        nv, nd, _ = sa.count_pairs(1, L, 2, 2, 128, S, T, [0, 2])
+        assert (nv, nd) == oracle.count_pairs(1, L, 2, 2, S, T, [0, 2])
+    # high positions: a window of 300 queries whose keys start one tail before it, against the same
+    # window moved down by a whole number of segments (the mask only depends on positions modulo S)
+    q0 = ((1 << 30) - 1 - 300) // S * S
+    lo = max(0, q0 - T)
+    hi = sa.count_pairs(1, 300, 2, 2, 128, S, T, [0, 2], kv_len=300 + q0 - lo, q_pos0=q0, kv_pos0=lo)
+    q1 = min(q0, 5 * S)
+    lo1 = max(0, q1 - T)
+    ref = sa.count_pairs(1, 300, 2, 2, 128, S, T, [0, 2], kv_len=300 + q1 - lo1, q_pos0=q1, kv_pos0=lo1)
+    assert hi[:2] == ref[:2]
+
+
 def test_unknown_head_class_is_rejected():
     with pytest.raises(sa.SegAttnError):
         sa.count_pairs(1, 256, 2, 2, 128, 64, 16, [0, 3])
