@@ -238,6 +238,42 @@ def test_empty_and_degenerate_shapes():
     assert torch.count_nonzero(dQ[:, 128:]) == 0
 
 
+def _random_case(rng):
+    d = int(rng.choice([64, 128]))
+    Hkv = int(rng.integers(1, 4))
+    g = int(rng.choice([1, 2, 4]))
+    S = int(rng.choice([int(rng.integers(1, 40)), int(rng.integers(40, 300)), 128, 256, int(rng.integers(300, 700))]))
+    T = int(rng.integers(0, S + 1)) if rng.random() < 0.8 else int(rng.choice([0, S]))
+    Lq = int(rng.integers(1, 900))
+    q0 = int(rng.integers(0, 4 * S + 1)) if rng.random() < 0.5 else 0
+    # keys from somewhere at or before the first query's tail (sometimes before position 0, sometimes too late)
+    k0 = q0 - int(rng.integers(0, 2 * S + 50)) if rng.random() < 0.8 else q0 + int(rng.integers(1, 100))
+    Lk = max(1, q0 + Lq - k0 - (int(rng.integers(0, 200)) if rng.random() < 0.3 else 0))
+    mask = [int(rng.integers(0, 3)) for _ in range(Hkv)]
+    X = int(rng.integers(0, q0 + Lq + 1)) if rng.random() < 0.4 else 0
+    return dict(B=int(rng.integers(1, 3)), Lq=Lq, Lk=Lk, Hq=Hkv * g, Hkv=Hkv, d=d, S=S, T=T, q0=q0, k0=k0, mask=mask,
+                X=X, tail_sg=bool(rng.random() < 0.3))
+
+
+@pytest.mark.parametrize("seed", range(64))
+def test_random_shapes_offsets_classes_and_boundaries(seed):
+    # seeded random problems over everything the interface takes at once: ragged sizes, position offsets on
+    # both sides (keys starting before position 0 or after the first query), head classes, the paper-literal
+    # flag and a detached prefix
+    c = _random_case(np.random.default_rng(1000 + seed))
+    Q, K, V, dO = rand_inputs(c["B"], c["Lq"], c["Hq"], c["Hkv"], c["d"], seed=seed, Lk=c["Lk"])
+    kw = dict(q_pos0=c["q0"], kv_pos0=c["k0"])
+    O, LSE = sa.seg_attn_fwd(Q, K, V, c["S"], c["T"], c["mask"], **kw)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, c["S"], c["T"], c["mask"], flagged_tail_is_sg=c["tail_sg"],
+                                 detach_before=c["X"], **kw)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), c["S"], c["T"], c["mask"], **kw)
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), c["S"], c["T"], c["mask"], flagged_tail_is_sg=c["tail_sg"],
+                     detach_before=c["X"], **kw)
+    assert_fwd_close(O, LSE, Oo, LSEo, "fwd %r" % c)
+    assert_grads_close((dQ, dK, dV), ref, "bwd %r" % c)
+
+
 def test_limits_of_the_interface():
     # 64 KV heads (the most the head table holds), all three classes, one query head each
     Hkv = 64
