@@ -78,3 +78,57 @@ def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0,
             dK[b, :, c] += scale * ((dS * dif).T @ Q[b, :, h])
             dV[b, :, c] += (P * dif).T @ dO[b, :, h]
     return dQ, dK, dV
+
+
+def retrieved_context(K_pool, V_pool, idx, K_seg, V_seg):
+    """Keys and values a head with a retrieved prefix attends over: ``[K_ret ; K_i]`` with
+    ``K_ret[b, r, c] = K_pool[b, idx[b, c, r], c]`` (Appendix C, Eq. "ctx", first case).  Shapes:
+    pools ``[B, P, Hkv, d]``, ``idx [B, Hkv, R]``, segment ``[B, Lseg, Hkv, d]`` -> ``[B, R + Lseg, Hkv, d]``."""
+    K_pool, V_pool, K_seg, V_seg = (np.asarray(x) for x in (K_pool, V_pool, K_seg, V_seg))
+    idx = np.asarray(idx)
+    B, Hkv, R = idx.shape
+    out = []
+    for pool, seg in ((K_pool, K_seg), (V_pool, V_seg)):
+        ctx = np.empty((B, R + seg.shape[1], Hkv, pool.shape[3]), dtype=pool.dtype)
+        for b in range(B):
+            for c in range(Hkv):
+                for r in range(R):
+                    ctx[b, r, c] = pool[b, idx[b, c, r], c]
+        ctx[:, R:] = seg
+        out.append(ctx)
+    return out[0], out[1]
+
+
+def retrieved_attention(Q_seg, K_pool, V_pool, idx, K_seg, V_seg, dO=None, scale=None):
+    """Attention of one segment over ``[retrieved prefix ; own segment]``: every prefix row visible, the
+    segment causal (Appendix C, Eq. "attn"); the prefix is stop-gradient (Definition 3.2, Lemma B.1).
+    Returns (O, LSE) or, with dO, (O, LSE, dQ, dK_seg, dV_seg)."""
+    Kc, Vc = retrieved_context(K_pool, V_pool, idx, K_seg, V_seg)
+    Q = np.asarray(Q_seg, dtype=np.float64)
+    Kc, Vc = Kc.astype(np.float64), Vc.astype(np.float64)
+    B, L, Hq, d = Q.shape
+    Hkv, R = Kc.shape[2], Kc.shape[1] - L
+    g = Hq // Hkv
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    vis = np.concatenate([np.ones((L, R), bool), np.tril(np.ones((L, L), bool))], axis=1)
+    O, LSE = np.zeros_like(Q), np.zeros((B, Hq, L))
+    dQ = np.zeros_like(Q)
+    dK, dV = np.zeros((B, L, Hkv, d)), np.zeros((B, L, Hkv, d))
+    for b in range(B):
+        for h in range(Hq):
+            c = h // g
+            s = np.where(vis, scale * (Q[b, :, h] @ Kc[b, :, c].T), -np.inf)
+            m = s.max(axis=1, keepdims=True)
+            e = np.exp(s - m)
+            z = e.sum(axis=1, keepdims=True)
+            P = e / z
+            O[b, :, h] = P @ Vc[b, :, c]
+            LSE[b, h] = (m + np.log(z))[:, 0]
+            if dO is not None:
+                go = np.asarray(dO, dtype=np.float64)[b, :, h]
+                dP = go @ Vc[b, :, c].T
+                dS = P * (dP - (go * O[b, :, h]).sum(axis=1, keepdims=True))
+                dQ[b, :, h] = scale * dS @ Kc[b, :, c]
+                dK[b, :, c] += scale * dS[:, R:].T @ Q[b, :, h]   # the segment's own keys only
+                dV[b, :, c] += P[:, R:].T @ go
+    return (O, LSE) if dO is None else (O, LSE, dQ, dK, dV)

@@ -217,6 +217,57 @@ def test_windows_with_detached_incoming_state_compose_to_depth_one_truncation():
         np.testing.assert_allclose(a, b, atol=TOL)
 
 
+# ---- retrieved prefix: [K_ret ; K_i] -------------------------------------------------------------
+def test_retrieving_every_older_position_is_the_dense_past_access_head():
+    # with the index list naming all positions before the segment, the retrieved context is the context of a
+    # past-access head of the dense reading; its own-segment gradients are those of that head too
+    L, S = 96, 32
+    Q, K, V, dO = rand(2, L, 4, 2, 8)
+    O, LSE = oracle.fwd(Q, K, V, S, 0, head_past_mask=[1, 1])
+    for i in range(1, L // S):
+        sl = slice(i * S, (i + 1) * S)
+        idx = np.broadcast_to(np.arange(i * S, dtype=np.int32), (2, 2, i * S))
+        dOw = np.zeros_like(dO)
+        dOw[:, sl] = dO[:, sl]
+        _, dK, dV = oracle.bwd(Q, K, V, dOw, S, 0, head_past_mask=[1, 1])
+        dQ = oracle.bwd(Q, K, V, dOw, S, 0, head_past_mask=[1, 1])[0]
+        o, lse, gq, gk, gv = dense.retrieved_attention(Q[:, sl], K, V, idx, K[:, sl], V[:, sl], dO[:, sl])
+        np.testing.assert_allclose(o, O[:, sl], atol=TOL)
+        np.testing.assert_allclose(lse, LSE[:, :, sl], atol=TOL)
+        np.testing.assert_allclose(gq, dQ[:, sl], atol=TOL)
+        np.testing.assert_allclose(gk, dK[:, sl], atol=TOL)     # T = 0: only the own segment is differentiable
+        np.testing.assert_allclose(gv, dV[:, sl], atol=TOL)
+
+
+def test_retrieved_prefix_is_order_free_and_matches_library_attention():
+    rng = np.random.default_rng(3)
+    Q, Kp, Vp, dO = rand(1, 40, 2, 2, 8, rng)
+    Ks, Vs = rng.standard_normal((1, 12, 2, 8)), rng.standard_normal((1, 12, 2, 8))
+    Qs, dOs = Q[:, :12], dO[:, :12]
+    idx = np.stack([rng.choice(40, size=9, replace=False) for _ in range(2)])[None].astype(np.int32)
+    Kc, Vc = dense.retrieved_context(Kp, Vp, idx, Ks, Vs)
+    for c in range(2):
+        np.testing.assert_array_equal(Kc[0, :9, c], Kp[0, idx[0, c], c])
+        np.testing.assert_array_equal(Vc[0, 9:, c], Vs[0, :, c])
+    o1, l1 = dense.retrieved_attention(Qs, Kp, Vp, idx, Ks, Vs)
+    o2, l2 = dense.retrieved_attention(Qs, Kp, Vp, idx[:, :, ::-1], Ks, Vs)   # softmax does not see the order
+    np.testing.assert_allclose(o1, o2, atol=TOL)
+    np.testing.assert_allclose(l1, l2, atol=TOL)
+    # library attention over the same context with the same mask, prefix detached
+    q = t64(Qs, True)
+    ks, vs = t64(Ks, True), t64(Vs, True)
+    kc = torch.cat([t64(Kc[:, :9]), ks], dim=1)
+    vc = torch.cat([t64(Vc[:, :9]), vs], dim=1)
+    m = torch.cat([torch.ones(12, 9, dtype=torch.bool), torch.ones(12, 12, dtype=torch.bool).tril()], dim=1)
+    o = F.scaled_dot_product_attention(q.transpose(1, 2), kc.transpose(1, 2), vc.transpose(1, 2), attn_mask=m).transpose(1, 2)
+    (o * t64(dOs)).sum().backward()
+    o3, _, gq, gk, gv = dense.retrieved_attention(Qs, Kp, Vp, idx, Ks, Vs, dOs)
+    np.testing.assert_allclose(o3, o.detach().numpy(), atol=TOL)
+    np.testing.assert_allclose(gq, q.grad.numpy(), atol=TOL)
+    np.testing.assert_allclose(gk, ks.grad.numpy(), atol=TOL)
+    np.testing.assert_allclose(gv, vs.grad.numpy(), atol=TOL)
+
+
 # ---- closed form: zero keys => uniform attention over the visible set ---------------------------
 def test_zero_keys_closed_form_counts_the_context():
     B, L, Hq, Hkv, d, S, T = 1, 120, 2, 2, 4, 40, 10
