@@ -172,6 +172,26 @@ segattn_status seg_prefill_step(seg_prefill_handle* h, const void* Qseg, const v
 segattn_status seg_prefill_reset(seg_prefill_handle* h); /* back to segment 0; state contents become dead */
 void seg_prefill_destroy(seg_prefill_handle* h);
 
+/* ---- Context of a head that reads a retrieved prefix (Appendix C, Eq. "ctx", first case: a
+ * long-range head in a long-range layer attends over [K_ret ; K_i], R retrieved rows followed by
+ * its own segment; Appendix D fixes R positions per head).  Given the R positions, builds
+ *     K_ctx[b][r][c][:]     = K_pool[b][idx[b][c][r]][c][:]      0 <= r < R
+ *     K_ctx[b][R + t][c][:] = K_seg[b][t][c][:]                  0 <= t < Lseg
+ * and V_ctx alike.  K_pool/V_pool are bf16 with element strides pool_stride (batch, position, head)
+ * and pool_len positions; K_seg/V_seg likewise with seg_stride; K_ctx/V_ctx are contiguous
+ * [B][R + Lseg][Hkv][d].  idx is a DEVICE array of int32, [B][Hkv][R].  All pointers 16-byte
+ * aligned, strides multiples of 8.  An index outside [0, pool_len) is not read: its row is zero
+ * and the next seg_attn_poll_status returns SEGATTN_ERR_INVALID.  The attention itself is the
+ * existing entry points on the context: seg_attn_fwd / seg_attn_bwd with Lq = Lseg, kv_len = R + Lseg,
+ * q_pos0 = R, kv_pos0 = 0, S = R + Lseg, T = 0, class 0 heads, and, in the backward,
+ * detach_before = R (the retrieved rows are forward-only: Definition 3.2, Lemma B.1); rows
+ * [R, R + Lseg) of the dK/dV it returns are the segment's gradients.  Choosing the R positions
+ * (the scoring and top-k selection of Appendix D) is not part of this library. */
+segattn_status seg_attn_gather_context(int32_t B, int32_t Hkv, int32_t d, int32_t R, int32_t Lseg, int32_t pool_len,
+                                       const void* K_pool, const void* V_pool, const int64_t pool_stride[3],
+                                       const void* K_seg, const void* V_seg, const int64_t seg_stride[3],
+                                       const int32_t* idx, void* K_ctx, void* V_ctx, void* stream);
+
 /* ---- Whole training-step call with HOST buffers (pinned or pageable): copies Q, K, V, dO to
  * the device arena, runs forward and backward, copies O, LSE, dQ, dK, dV back, and
  * synchronises `stream` before returning.  Host tensors are contiguous in the layouts
@@ -189,7 +209,8 @@ segattn_status seg_attn_step_host(const seg_attn_params* p, const void* Q_host, 
 
 /* ---- Status and accounting */
 /* Synchronises `stream`, then reads and clears the device status word that kernels set when a
- * bounded wait expires.  Returns SEGATTN_OK, SEGATTN_ERR_TIMEOUT or SEGATTN_ERR_CUDA. */
+ * bounded wait expires or a kernel refuses its input.  Returns SEGATTN_OK, SEGATTN_ERR_TIMEOUT,
+ * SEGATTN_ERR_INVALID (an index out of range in seg_attn_gather_context) or SEGATTN_ERR_CUDA. */
 segattn_status seg_attn_poll_status(void* stream);
 const char* seg_attn_status_string(segattn_status s);
 /* Last CUDA error code (cudaError_t or CUresult as int) recorded by this thread's failing call. */

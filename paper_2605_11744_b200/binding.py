@@ -62,6 +62,8 @@ def lib():
         L.seg_attn_profile_kernels.argtypes = [pp, vp, vp, vp, vp, fp, vp, u8p, vp, vp, vp, vp, ctypes.c_size_t,
                                                ctypes.c_int, ctypes.POINTER(ctypes.c_float * 4), vp]
         L.seg_attn_poll_status.argtypes = [vp]
+        L.seg_attn_gather_context.argtypes = [ctypes.c_int32] * 6 + [vp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp,
+                                                                     ctypes.POINTER(ctypes.c_int64), vp, vp, vp, vp]
         L.seg_attn_selftest_wait_timeout.argtypes = [vp]
         L.seg_attn_status_string.restype = ctypes.c_char_p
         L.seg_attn_status_string.argtypes = [ctypes.c_int]
@@ -214,6 +216,26 @@ def seg_attn_step_host(Q, K, V, dO, S: int, T: int, head_past_mask=None, sm_scal
                                     ctypes.c_void_p(arena.data_ptr()), arena.numel(), _stream(stream)),
            "seg_attn_step_host")
     return outs
+
+
+def gather_context(K_pool, V_pool, idx, K_seg, V_seg, stream=None):
+    """[retrieved rows ; segment rows] for K and V - the C entry point `seg_attn_gather_context`.
+    K_pool, V_pool [B, P, Hkv, d]; idx int32 [B, Hkv, R] (device); K_seg, V_seg [B, Lseg, Hkv, d]."""
+    _need_cuda_bf16(K_pool, V_pool, K_seg, V_seg)
+    if idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous():
+        raise ValueError("idx must be a contiguous int32 CUDA tensor")
+    B, P, Hkv, d = K_pool.shape
+    R, Lseg = idx.shape[2], K_seg.shape[1]
+    if idx.shape[:2] != (B, Hkv) or K_seg.shape[0] != B or K_seg.shape[2:] != (Hkv, d):
+        raise ValueError("shapes do not fit")
+    if V_pool.stride() != K_pool.stride() or V_seg.stride() != K_seg.stride():
+        raise ValueError("K and V must share strides")
+    K_ctx = torch.empty((B, R + Lseg, Hkv, d), dtype=torch.bfloat16, device=K_pool.device)
+    V_ctx = torch.empty_like(K_ctx)
+    _check(lib().seg_attn_gather_context(B, Hkv, d, R, Lseg, P, _ptr(K_pool), _ptr(V_pool), _strides3(K_pool),
+                                         _ptr(K_seg), _ptr(V_seg), _strides3(K_seg), _ptr(idx), _ptr(K_ctx),
+                                         _ptr(V_ctx), _stream(stream)), "seg_attn_gather_context")
+    return K_ctx, V_ctx
 
 
 def profile_kernels(Q, K, V, dO, S: int, T: int, head_past_mask=None, sm_scale=None, iters: int = 5, stream=None):

@@ -57,4 +57,48 @@ __global__ void __launch_bounds__(256) prefill_roll_tail_kernel(uint4* Kwin, uin
     Vwin[base + off] = Vwin[base + (long long)S * d16 + off];
 }
 
+// Context of a head that reads a retrieved prefix (Appendix C, Eq. "ctx", first case): rows [0, R) of
+// the output are the pool rows the index list names, rows [R, R + Lseg) the current segment's.  One
+// thread per 16 bytes of output (K and V both).  An index outside [0, pool_len) gives a zero row and
+// sets the status word (code 1, invalid input) instead of reading out of bounds.
+struct GatherParams {
+    const uint4* Kpool;  // strides below, in uint4 units, for (batch, position, head)
+    const uint4* Vpool;
+    const uint4* Kseg;
+    const uint4* Vseg;
+    const int32_t* idx;  // [B][Hkv][R]
+    uint4* Kctx;         // [B][R + Lseg][Hkv][d], contiguous
+    uint4* Vctx;
+    long long pool_stride[3], seg_stride[3];
+    int B, Hkv, R, Lseg, pool_len;
+    int d16;             // d * 2 / 16
+};
+__global__ void __launch_bounds__(256) gather_context_kernel(const GatherParams prm, int* status) {
+    const int rows = prm.R + prm.Lseg;
+    const long long n = (long long)prm.B * rows * prm.Hkv * prm.d16;
+    const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    const int e = (int)(i % prm.d16);
+    const int h = (int)((i / prm.d16) % prm.Hkv);
+    const int r = (int)((i / ((long long)prm.d16 * prm.Hkv)) % rows);
+    const int b = (int)(i / ((long long)prm.d16 * prm.Hkv * rows));
+    uint4 k = make_uint4(0, 0, 0, 0), v = k;
+    if (r < prm.R) {
+        const int j = prm.idx[((long long)b * prm.Hkv + h) * prm.R + r];
+        if (j >= 0 && j < prm.pool_len) {
+            const long long src = b * prm.pool_stride[0] + (long long)j * prm.pool_stride[1] + h * prm.pool_stride[2] + e;
+            k = prm.Kpool[src];
+            v = prm.Vpool[src];
+        } else if (e == 0) {
+            atomicCAS(status, 0, (1 << 8) | 1);
+        }
+    } else {
+        const long long src = b * prm.seg_stride[0] + (long long)(r - prm.R) * prm.seg_stride[1] + h * prm.seg_stride[2] + e;
+        k = prm.Kseg[src];
+        v = prm.Vseg[src];
+    }
+    prm.Kctx[i] = k;
+    prm.Vctx[i] = v;
+}
+
 }  // namespace segattn

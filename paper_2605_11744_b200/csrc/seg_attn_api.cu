@@ -264,7 +264,8 @@ segattn_status seg_attn_poll_status(void* stream) {
     int zero = 0;
     e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
     if (e != cudaSuccess) return cuda_fail(e);
-    return SEGATTN_ERR_TIMEOUT;
+    // the word is (status << 8) | detail: an expired wait, or input a kernel refused (an index out of range)
+    return (word >> 8) == SEGATTN_ERR_INVALID ? SEGATTN_ERR_INVALID : SEGATTN_ERR_TIMEOUT;
 }
 
 const char* seg_attn_status_string(segattn_status s) {

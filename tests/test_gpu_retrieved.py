@@ -1,0 +1,75 @@
+"""Attention over a retrieved prefix on the GPU: the gather is exact, and the existing forward and
+backward on the gathered context match the oracle's [K_ret ; K_i] attention."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dense
+import paper_2605_11744_b200 as sa
+from util import assert_fwd_close, assert_grads_close, f64
+
+pytestmark = pytest.mark.gpu
+
+
+def bits(t):
+    return t.contiguous().view(torch.int16).cpu().numpy()
+
+
+def make(B, P, Hq, Hkv, d, R, Lseg, seed, pool_layout="blhd"):
+    g = torch.Generator().manual_seed(seed)
+    mk = lambda *s: torch.randn(*s, generator=g).bfloat16().cuda()
+    if pool_layout == "blhd":
+        Kp, Vp = mk(B, P, Hkv, d), mk(B, P, Hkv, d)
+    else:  # the layout of a per-head pool, [B][Hkv][P][d], seen as [B, P, Hkv, d]
+        Kp, Vp = mk(B, Hkv, P, d).permute(0, 2, 1, 3), mk(B, Hkv, P, d).permute(0, 2, 1, 3)
+    idx = torch.randint(0, P, (B, Hkv, R), generator=g, dtype=torch.int32).cuda()
+    return Kp, Vp, idx, mk(B, Lseg, Hkv, d), mk(B, Lseg, Hkv, d), mk(B, Lseg, Hq, d), mk(B, Lseg, Hq, d)
+
+
+@pytest.mark.parametrize("B,P,Hq,Hkv,d,R,Lseg,layout", [
+    (1, 2048, 4, 2, 128, 512, 512, "blhd"),     # R = 512 as in the paper's setting, several tiles
+    (2, 1000, 4, 4, 128, 300, 200, "bhld"),     # nothing aligned to a tile; pool stored per head
+    (1, 700, 2, 1, 64, 129, 77, "blhd"),        # d = 64, ragged
+    (2, 64, 2, 2, 128, 0, 256, "blhd"),         # nothing retrieved: plain causal attention of the segment
+    (1, 512, 2, 2, 128, 256, 1, "bhld"),        # a single query row
+])
+def test_retrieved_prefix_attention_matches_oracle(B, P, Hq, Hkv, d, R, Lseg, layout):
+    Kp, Vp, idx, Ks, Vs, Q, dO = make(B, P, Hq, Hkv, d, R, Lseg, seed=P + R, pool_layout=layout)
+    Kc, Vc = sa.gather_context(Kp, Vp, idx, Ks, Vs)
+    sa.poll_status()
+    # index work: bit-exact against the oracle's gather
+    Kc_ref, Vc_ref = dense.retrieved_context(bits(Kp), bits(Vp), idx.cpu().numpy(), bits(Ks), bits(Vs))
+    assert np.array_equal(bits(Kc), Kc_ref) and np.array_equal(bits(Vc), Vc_ref)
+    # the attention is the library's forward / backward on the context: queries at positions R.., one
+    # segment, and the retrieved rows detached
+    S = max(1, R + Lseg)
+    mask = [0] * Hkv
+    O, LSE = sa.seg_attn_fwd(Q, Kc, Vc, S, 0, mask, q_pos0=R, kv_pos0=0)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, Kc, Vc, O, LSE, dO, S, 0, mask, q_pos0=R, kv_pos0=0, detach_before=R)
+    sa.poll_status()
+    Oo, LSEo, gq, gk, gv = dense.retrieved_attention(f64(Q), f64(Kp), f64(Vp), idx.cpu().numpy(), f64(Ks), f64(Vs), f64(dO))
+    assert_fwd_close(O, LSE, Oo, LSEo, "retrieved prefix")
+    assert_grads_close((dQ, dK[:, R:], dV[:, R:]), (gq, gk, gv), "retrieved prefix")
+    assert not dK[:, :R].any() and not dV[:, :R].any()
+
+
+def test_an_index_out_of_range_is_reported_and_not_read():
+    Kp, Vp, idx, Ks, Vs, _, _ = make(1, 100, 2, 2, 128, 16, 8, seed=9)
+    idx[0, 1, 3] = 100
+    idx[0, 0, 5] = -1
+    Kc, Vc = sa.gather_context(Kp, Vp, idx, Ks, Vs)
+    with pytest.raises(sa.SegAttnError) as e:
+        sa.poll_status()
+    assert e.value.status == 1
+    sa.poll_status()   # cleared
+    assert not Kc[0, 3, 1].any() and not Vc[0, 5, 0].any()
+    ok = idx.clone()
+    ok[0, 1, 3] = 0
+    ok[0, 0, 5] = 0
+    Kc2, _ = sa.gather_context(Kp, Vp, ok, Ks, Vs)
+    sa.poll_status()
+    keep = torch.ones(16 + 8, 2, dtype=torch.bool)
+    keep[3, 1] = keep[5, 0] = False
+    assert torch.equal(Kc[0][keep.cuda()], Kc2[0][keep.cuda()])
+    with pytest.raises(sa.SegAttnError):
+        sa.gather_context(Kp[:, :, :, :100], Vp[:, :, :, :100], idx, Ks[:, :, :, :100], Vs[:, :, :, :100])   # d = 100
