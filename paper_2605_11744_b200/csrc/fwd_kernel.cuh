@@ -210,66 +210,76 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         // The two kinds of product are issued by two warps on different schedulers, so that neither
         // waits behind the other's barriers and each has half the issue work.
         constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
-        long long g = 0;  // key tiles of earlier work items
+        static_assert(NV == 2 && NK == 2 && NQ == 1, "ring indices below are written out for these depths");
+        int g = 0;  // key tiles of earlier work items (a CTA sees far fewer than 2^31)
         bool ok = true;
         ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
+        // The chain P(j) written -> PV(j) issued -> PV(j) finished -> S(j+3) issued -> S(j+3) finished sets
+        // the pace of the kernel, so what the two issuers execute between a barrier and their first product
+        // is kept short: everything that does not depend on the barrier is worked out before the wait, the
+        // waits of one batch share one vote, and optional completion signals are predicated.
         for (int item; ok && walk.next(&item);) {
             const FwdItem it = fwd_decode(prm, item);
             int t_lo, n;
             fwd_item_tiles(prm, it, &t_lo, &n);
             if (n == 0) continue;
-            for (int j = 0; ok && j < n; ++j) {
-                const long long gj = g + j;
-                const int sv = (int)(gj % NV);
-                ok = warp_wait(bar(kBarVFull + sv), (uint32_t)((gj / NV) & 1), 6) &&
-                     warp_wait(bar(kBarPFull + (int)(gj & 1)), (uint32_t)((gj >> 1) & 1), 7);
-                if (!ok) break;
+            for (int j = 0; j < n; ++j) {
+                const int gj = g + j;
+                const int sv = gj & 1;
+                const uint32_t ph = (uint32_t)(gj >> 1) & 1;
+                const uint32_t a_p = tS0 + (uint32_t)(gj % 3) * 128;
+                const uint32_t b_free = bar(kBarSFree + gj % 3);
+                const uint64_t vd = make_sdesc(sV(sv), 16384, 1024);
+                // V tile landed, P written (the two barriers share ring position and phase)
+                if (!(ok = warp_wait2(bar(kBarVFull + sv), ph, bar(kBarPFull + sv), ph, 6))) break;
                 tc_fence_after();
                 TRACE(lane == 0, j * 8 + 4);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
-                    mma_ts(tO, tS(gj) + k * 8, make_sdesc(sV(sv) + k * 2048, 16384, 1024), idesc_pv, (j > 0) || (k > 0));
+                    mma_ts(tO, a_p + k * 8, vd + ((k * 2048) >> 4), idesc_pv, (j > 0) || (k > 0));
+                mma_commit(b_free);  // first: P(j) is consumed, the S buffer may take new scores
                 mma_commit(bar(kBarVEmpty + sv));
-                mma_commit(bar(kBarPvDone + (int)(gj & 1)));
-                mma_commit(bar(kBarSFree + (int)(gj % 3)));  // P(j) is consumed: the S buffer may take new scores
+                mma_commit(bar(kBarPvDone + sv));
+                mma_commit_if(j == n - 1, bar(kBarOFull));  // the item's O is complete
                 TRACE(lane == 0, j * 8 + 5);
             }
-            if (ok) mma_commit(bar(kBarOFull));  // the item's O is complete
             g += n;
         }
     } else if (warp == 2) {
         // ---------------- MMA issuer for S = Q K^T (whole warp; one elected lane issues) ----------------
         constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
-        int qn = 0;       // work items with visible tiles started so far
-        long long g = 0;  // key tiles of earlier work items
+        int qn = 0;  // work items with visible tiles started so far
+        int g = 0;   // key tiles of earlier work items
         bool ok = true;
+        const uint64_t qd = make_sdesc(sQ(0), 16, 1024);
         ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
         for (int item; ok && walk.next(&item);) {
             const FwdItem it = fwd_decode(prm, item);
             int t_lo, n;
             fwd_item_tiles(prm, it, &t_lo, &n);
             if (n == 0) continue;
-            const int qs = qn % NQ;
-            if (!(ok = warp_wait(bar(kBarQFull + qs), (qn / NQ) & 1, 4))) break;
+            if (!(ok = warp_wait(bar(kBarQFull), (uint32_t)qn & 1, 4))) break;
             ++qn;
-            for (int j = 0; ok && j < n; ++j) {
-                const long long gj = g + j;
-                // the S buffer of tile gj held P of tile gj - 3: wait until that PV product has finished
-                if (gj >= 3) {
-                    ok = warp_wait(bar(kBarSFree + (int)(gj % 3)), (uint32_t)(((gj - 3) / 3) & 1), 12);
-                    if (!ok) break;
-                    tc_fence_after();
-                }
-                const int s = (int)(gj % NK);
-                if (!(ok = warp_wait(bar(kBarKFull + s), (uint32_t)((gj / NK) & 1), 5))) break;
+            for (int j = 0; j < n; ++j) {
+                const int gj = g + j;
+                const int s = gj & 1;
+                const int s3 = gj % 3;
+                const uint32_t d_s = tS0 + (uint32_t)s3 * 128;
+                const uint64_t kd = make_sdesc(sK(s), 16, 1024);
+                // The S buffer of tile gj held P of tile gj - 3: that PV product has finished (the first
+                // three tiles of a launch find fresh buffers: parity 1 of a new barrier reads complete);
+                // and the K tile has landed.
+                const uint32_t free_ph = gj >= 3 ? (uint32_t)((gj - 3) / 3) & 1 : 1u;
+                if (!(ok = warp_wait2(bar(kBarSFree + s3), free_ph, bar(kBarKFull + s), (uint32_t)(gj >> 1) & 1, 12))) break;
+                tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-                    mma_ss(tS(gj), make_sdesc(sQ(qs) + off, 16, 1024), make_sdesc(sK(s) + off, 16, 1024), idesc_qk, k > 0);
+                    const uint32_t off = ((k / 4) * 16384 + (k % 4) * 32) >> 4;  // descriptor addresses count 16-byte units
+                    mma_ss(d_s, qd + off, kd + off, idesc_qk, k > 0);
                 }
+                mma_commit(bar(kBarSFull + s3));  // first: a softmax group waits for it
                 mma_commit(bar(kBarKEmpty + s));
-                mma_commit(bar(kBarSFull + (int)(gj % 3)));
-                if (j == n - 1) mma_commit(bar(kBarQEmpty + qs));  // the item's last scores release Q
+                mma_commit_if(j == n - 1, bar(kBarQEmpty));  // the item's last scores release Q
                 TRACE(lane == 0, j * 8 + 6);
             }
             g += n;
