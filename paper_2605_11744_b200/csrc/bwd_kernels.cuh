@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             int qn = 0;       // work items with visible tiles started so far
-            long long g = 0;  // key tiles requested so far (all work items)
+            int g = 0;  // key tiles requested so far (all work items; far fewer than 2^31)
             bool ok = true;
             ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items_dq);
         for (int item; ok && walk.next(&item);) {
@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                     tma_load_4d(sDO + pnl * 16384, &prm.tdo, bar(kBarDoFull), pnl * 64, it.hq, r0, it.b);
                 ++qn;
                 for (int j = 0; ok && j < n; ++j) {
-                    const long long gj = g + j;
+                    const int gj = g + j;
                     const int sk = (int)(gj % NK), sv = (int)(gj % NV);
                     const int row = (t_lo + j) * kTile;
                     if (!(ok = mbar_wait(bar(kBarKEmpty + sk), (uint32_t)((gj / NK) & 1) ^ 1, 11))) break;
@@ -309,7 +309,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
         const uint64_t sl2x2 = f32x2(sl2, sl2);
         constexpr int DH = D / 2;  // this thread's share of the row
         int qn = 0;
-        long long g = 0;  // key tiles of earlier work items
+        int g = 0;  // key tiles of earlier work items
         bool ok = true;
         ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items_dq);
         for (int item; ok && walk.next(&item);) {
@@ -386,7 +386,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                 }
             };
             for (int j = 0; j < n_tiles; ++j) {
-                const long long gj = g + j;
+                const int gj = g + j;
                 const uint32_t tS = tS0 + (uint32_t)(gj & 1) * 128;
                 const int c0 = (t_lo + j) * kTile;
                 const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);

@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     const uint32_t tS0 = tmem, tO = tmem + 384;
-    auto tS = [&](long long gj) { return tS0 + (uint32_t)(gj % 3) * 128; };  // S buffer of global key tile gj
+    auto tS = [&](int gj) { return tS0 + (uint32_t)(gj % 3) * 128; };  // S buffer of global key tile gj
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     return;
                 }
             };
-            long long g = 0;  // key tiles requested so far (all work items)
+            int g = 0;  // key tiles requested so far (all work items; far fewer than 2^31)
             advance_q();
             ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
         for (int item; ok && walk.next(&item);) {
@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 fwd_item_tiles(prm, it, &t_lo, &n);
                 if (n == 0) continue;
                 auto load_k = [&](int j) -> bool {
-                    const long long gj = g + j;
+                    const int gj = g + j;
                     const int s = (int)(gj % NK);
                     if (!mbar_wait(bar(kBarKEmpty + s), (uint32_t)((gj / NK) & 1) ^ 1, 2)) return false;
                     mbar_expect_tx(bar(kBarKFull + s), SM::kTileBytes);
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     return true;
                 };
                 auto load_v = [&](int j) -> bool {
-                    const long long gj = g + j;
+                    const int gj = g + j;
                     const int s = (int)(gj % NV);
                     if (!mbar_wait(bar(kBarVEmpty + s), (uint32_t)((gj / NV) & 1) ^ 1, 3)) return false;
                     mbar_expect_tx(bar(kBarVFull + s), SM::kTileBytes);
@@ -296,8 +296,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         constexpr int DH = D / 2;  // this group's share of an O row in the epilogue
         const float sl2 = prm.scale_log2;
         const uint64_t sl2x2 = f32x2(sl2, sl2);
-        long long g = 0;  // key tiles of earlier work items
-        int qn = 0;       // earlier work items that had visible tiles
+        int g = 0;   // key tiles of earlier work items (a CTA sees far fewer than 2^31)
+        int qn = 0;  // earlier work items that had visible tiles
         bool ok = true;
         ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
         for (int item; ok && walk.next(&item);) {
@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             TRACE(tid == 128, 2048 + qn * 4 + 0);
             // One key tile of the online softmax.  MASKED is a compile-time flag so that the common,
             // fully visible tile runs straight-line code.
-            auto softmax_tile = [&](auto masked_c, const int j, const long long gj, const int c0) {
+            auto softmax_tile = [&](auto masked_c, const int j, const int gj, const int c0) {
                 constexpr bool MASKED = decltype(masked_c)::value;
                 const uint32_t tSj = tS(gj);
                 uint32_t va[32], vb[32];
@@ -433,8 +433,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 }
             };
             for (int j = 0; j < n_tiles; ++j) {
-                const long long gj = g + j;
-                if ((int)(gj & 1) != grp) continue;  // the other group's tile
+                const int gj = g + j;
+                if ((gj & 1) != grp) continue;  // the other group's tile
                 const int c0 = (t_lo + j) * kTile;
                 const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
                 ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (int)(gj % 3)), (uint32_t)((gj / 3) & 1), 8));
