@@ -23,37 +23,62 @@ constexpr int kEwWarps = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ------------------------------------------------------------------------------------------
-// D[b][h][r] = sum_e dO[b][r][h][e] * O[b][r][h][e]; one group of D/8 threads per row, 16-byte loads.
+// D[b][h][r] = sum_e dO[b][r][h][e] * O[b][r][h][e]; one group of D/8 threads per row, 16-byte loads,
+// kRowdotUnroll rows per thread group with all their loads issued before the first is used (the kernel
+// is a pure stream: what matters is the number of bytes in flight per SM).
+constexpr int kRowdotUnroll = 4;
 template <int D>
 __global__ void __launch_bounds__(256) bwd_rowdot_kernel(const __nv_bfloat16* __restrict__ O,
                                                          const __nv_bfloat16* __restrict__ dO, float* __restrict__ Dvec,
                                                          int B, int Lq, int Hq, long long s0, long long s1,
                                                          long long s2) {
-    constexpr int TPR = D / 8;  // threads per row
+    constexpr int TPR = D / 8;          // threads per row
+    constexpr int RPB = 256 / TPR;      // rows a block covers per pass
     const long long n_rows = (long long)B * Lq * Hq;
-    const long long row = (long long)blockIdx.x * (256 / TPR) + threadIdx.x / TPR;
+    const long long row0 = (long long)blockIdx.x * (RPB * kRowdotUnroll) + threadIdx.x / TPR;
     const int part = threadIdx.x % TPR;
-    float acc = 0.f;
-    int b = 0, r = 0, h = 0;
-    if (row < n_rows) {
-        h = (int)(row % Hq);
-        r = (int)((row / Hq) % Lq);
-        b = (int)(row / ((long long)Hq * Lq));
-        const long long off = b * s0 + (long long)r * s1 + h * s2 + part * 8;
-        const uint4 a = *reinterpret_cast<const uint4*>(O + off);
-        const uint4 g = *reinterpret_cast<const uint4*>(dO + off);
-        const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
-        const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g);
+    uint4 a[kRowdotUnroll], g[kRowdotUnroll];
+    long long out[kRowdotUnroll];
+#pragma unroll
+    for (int u = 0; u < kRowdotUnroll; ++u) {
+        const long long row = row0 + (long long)u * RPB;
+        a[u] = make_uint4(0, 0, 0, 0);
+        g[u] = a[u];
+        out[u] = -1;
+        if (row < n_rows) {
+            int h, b, r;
+            if (n_rows <= 0xffffffffLL) {   // 32-bit division is several times cheaper than 64-bit
+                const unsigned bh = (unsigned)row / (unsigned)Hq;   // (b, r)
+                h = (int)((unsigned)row - bh * (unsigned)Hq);
+                b = (int)(bh / (unsigned)Lq);
+                r = (int)(bh - (unsigned)b * (unsigned)Lq);
+            } else {
+                const long long bh = row / Hq;
+                h = (int)(row - bh * Hq);
+                b = (int)(bh / Lq);
+                r = (int)(bh - (long long)b * Lq);
+            }
+            const long long off = b * s0 + (long long)r * s1 + h * s2 + part * 8;
+            a[u] = *reinterpret_cast<const uint4*>(O + off);
+            g[u] = *reinterpret_cast<const uint4*>(dO + off);
+            out[u] = ((long long)b * Hq + h) * Lq + r;
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kRowdotUnroll; ++u) {
+        const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a[u]);
+        const __nv_bfloat162* pg = reinterpret_cast<const __nv_bfloat162*>(&g[u]);
+        float acc = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const float2 x = __bfloat1622float2(pa[i]), y = __bfloat1622float2(pg[i]);
             acc = fmaf(x.x, y.x, acc);
             acc = fmaf(x.y, y.y, acc);
         }
-    }
 #pragma unroll
-    for (int o = TPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (row < n_rows && part == 0) Dvec[((long long)b * Hq + h) * Lq + r] = acc;
+        for (int o = TPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (out[u] >= 0 && part == 0) Dvec[out[u]] = acc;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
