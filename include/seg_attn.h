@@ -169,6 +169,20 @@ segattn_status seg_prefill_create(const seg_attn_params* p, const uint8_t* head_
  * those rows), then rolls the tail.  Call once per segment, in order, on one stream. */
 segattn_status seg_prefill_step(seg_prefill_handle* h, const void* Qseg, const void* Kseg, const void* Vseg,
                                 void* Oseg, float* LSEseg, void* stream);
+/* Backward of the segment stepped last (the streamed form of training with truncation depth 1: a
+ * segment is run forward, its loss is differentiated, and credit stops where the carried state
+ * entered - definition of the K-truncated objective with K = 1).  Valid after seg_prefill_step and
+ * before the next one; the state still holds what that step attended over.  Qseg, Oseg, dOseg and
+ * dQseg are [B][S][Hq][d] with the strides given at creation, LSEseg as returned by the step.
+ * dKctx and dVctx are contiguous bf16 [B][T+S][Hkv][d]: the gradients of the key/value rows at
+ * global positions [i*S - T, i*S + S) - the previous segment's carried tail, then the segment itself
+ * (rows before position 0 are zero).  Older rows of past-access heads are read forward-only and get
+ * none.  The caller adds the first T rows to the previous segment's gradients.  `workspace`: DEVICE,
+ * 256-byte aligned, at least seg_prefill_bwd_workspace_bytes(h) bytes. */
+size_t seg_prefill_bwd_workspace_bytes(const seg_prefill_handle* h);
+segattn_status seg_prefill_step_bwd(seg_prefill_handle* h, const void* Qseg, const void* Oseg, const float* LSEseg,
+                                    const void* dOseg, void* dQseg, void* dKctx, void* dVctx, void* workspace,
+                                    size_t workspace_bytes, void* stream);
 segattn_status seg_prefill_reset(seg_prefill_handle* h); /* back to segment 0; state contents become dead */
 void seg_prefill_destroy(seg_prefill_handle* h);
 

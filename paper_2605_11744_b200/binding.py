@@ -53,6 +53,9 @@ def lib():
         L.seg_prefill_state_bytes.argtypes = [pp, u8p]
         L.seg_prefill_create.argtypes = [pp, u8p, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
         L.seg_prefill_step.argtypes = [vp, vp, vp, vp, vp, fp, vp]
+        L.seg_prefill_bwd_workspace_bytes.restype = ctypes.c_size_t
+        L.seg_prefill_bwd_workspace_bytes.argtypes = [vp]
+        L.seg_prefill_step_bwd.argtypes = [vp, vp, vp, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.seg_prefill_reset.argtypes = [vp]
         L.seg_prefill_destroy.argtypes = [vp]
         L.seg_prefill_destroy.restype = None
@@ -286,6 +289,25 @@ class Prefill:
         _check(lib().seg_prefill_step(self._h, _ptr(Qseg), _ptr(Kseg), _ptr(Vseg), _ptr(O), _ptr(LSE),
                                       _stream(stream)), "seg_prefill_step")
         return O, LSE
+
+    def step_bwd(self, Qseg, Oseg, LSEseg, dOseg, stream=None):
+        """Backward of the segment stepped last: dQ [B,S,Hq,d] and dK, dV [B,T+S,Hkv,d] for the key/value rows
+        [previous tail ; segment] - the C entry point `seg_prefill_step_bwd`."""
+        _need_cuda_bf16(Qseg, Oseg, dOseg)
+        p = self.params
+        for t in (Qseg, Oseg, dOseg):
+            if tuple(t.shape) != (p.B, p.S, p.Hq, p.d) or not t.is_contiguous():
+                raise ValueError("segment tensors must be contiguous [B,S,Hq,d]")
+        dQ = torch.empty_like(Qseg)
+        dK = torch.empty((p.B, p.T + p.S, p.Hkv, p.d), dtype=torch.bfloat16, device=Qseg.device)
+        dV = torch.empty_like(dK)
+        need = int(lib().seg_prefill_bwd_workspace_bytes(self._h))
+        if getattr(self, "_bwd_ws", None) is None or self._bwd_ws.numel() < need:
+            self._bwd_ws = torch.empty(max(need, 256), dtype=torch.uint8, device=Qseg.device)
+        _check(lib().seg_prefill_step_bwd(self._h, _ptr(Qseg), _ptr(Oseg), _ptr(LSEseg), _ptr(dOseg), _ptr(dQ), _ptr(dK),
+                                          _ptr(dV), ctypes.c_void_p(self._bwd_ws.data_ptr()), self._bwd_ws.numel(),
+                                          _stream(stream)), "seg_prefill_step_bwd")
+        return dQ, dK, dV
 
     def reset(self):
         _check(lib().seg_prefill_reset(self._h), "seg_prefill_reset")

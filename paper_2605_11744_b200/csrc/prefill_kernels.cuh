@@ -57,6 +57,31 @@ __global__ void __launch_bounds__(256) prefill_roll_tail_kernel(uint4* Kwin, uin
     Vwin[base + off] = Vwin[base + (long long)S * d16 + off];
 }
 
+// Gradients of the streamed backward, from the two per-class scratch tensors ([B][n][T+S][d], slot order)
+// to the caller's [B][T+S][Hkv][d]: one thread per 16 bytes (dK and dV both).
+__global__ void __launch_bounds__(256) prefill_scatter_grads_kernel(const PrefillCopyParams prm, const uint4* gKf,
+                                                                    const uint4* gVf, const uint4* gKu, const uint4* gVu,
+                                                                    uint4* dK, uint4* dV) {
+    const int rows = prm.T + prm.S;
+    const long long n = (long long)prm.B * rows * prm.Hkv * prm.d16;
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= n) return;
+    const int e = (int)(idx % prm.d16);
+    const int h = (int)((idx / prm.d16) % prm.Hkv);
+    const int r = (int)((idx / ((long long)prm.d16 * prm.Hkv)) % rows);
+    const int b = (int)(idx / ((long long)prm.d16 * prm.Hkv * rows));
+    const int slot = prm.slot_of_head[h];
+    if (prm.flag_of_head[h]) {
+        const long long src = (((long long)b * prm.n_flag + slot) * rows + r) * prm.d16 + e;
+        dK[idx] = gKf[src];
+        dV[idx] = gVf[src];
+    } else {
+        const long long src = (((long long)b * prm.n_unflag + slot) * rows + r) * prm.d16 + e;
+        dK[idx] = gKu[src];
+        dV[idx] = gVu[src];
+    }
+}
+
 // Context of a head that reads a retrieved prefix (Appendix C, Eq. "ctx", first case): rows [0, R) of
 // the output are the pool rows the index list names, rows [R, R + Lseg) the current segment's.  One
 // thread per 16 bytes of output (K and V both).  An index outside [0, pool_len) gives a zero row and

@@ -82,3 +82,47 @@ def test_configuration_4_streamed_at_full_size_sampled():
         ps = sorted(set(int(p) for p in rng.integers(0, w.L, size=10)) | {0, w.S - 1, w.S, w.L - 1})
         for p, Oo, LSEo, _ in oracle_rows(x, w, 0, c, hq, ps):
             assert_fwd_close(O[:, p:p + 1, hq], LSE[:, hq, p:p + 1], Oo, LSEo, "cfg4 row %d kv%d" % (p, c))
+
+
+@pytest.mark.parametrize("B,L,Hq,Hkv,d,S,T,mask", [
+    (1, 1024, 4, 2, 128, 256, 128, [0, 1]),
+    (2, 768, 4, 4, 128, 256, 0, [1, 0, 0, 1]),
+    (1, 800, 2, 2, 64, 200, 72, [0, 1]),
+    (1, 1024, 6, 3, 128, 256, 256, [2, 1, 0]),     # all head classes, tail = whole previous segment
+    (1, 512, 2, 1, 128, 128, 64, [1]),             # past-access heads only
+])
+def test_streamed_backward_sums_to_the_one_shot_backward(B, L, Hq, Hkv, d, S, T, mask):
+    # segment by segment: forward, then the backward of that segment's loss term; the key/value gradients of
+    # [previous tail ; segment] added up over the segments are those of the whole-sequence backward (one
+    # attention layer has no longer state chain than one transition), and every term matches the oracle
+    from util import assert_grads_close
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=L + S)
+    pf = sa.Prefill(B, S, T, Hq, Hkv, d, L, mask)
+    dQ = torch.empty_like(Q)
+    dK = torch.zeros(B, L, Hkv, d, dtype=torch.float32, device="cuda")
+    dV = torch.zeros_like(dK)
+    Qf, Kf, Vf, dOf = f64(Q), f64(K), f64(V), f64(dO)
+    for i in range(L // S):
+        sl = slice(i * S, (i + 1) * S)
+        q, do = Q[:, sl].contiguous(), dO[:, sl].contiguous()
+        o, lse = pf.step(q, K[:, sl].contiguous(), V[:, sl].contiguous())
+        gq, gk, gv = pf.step_bwd(q, o, lse, do)
+        sa.poll_status()
+        dQ[:, sl] = gq
+        lo = i * S - T
+        cut = max(0, -lo)
+        assert not gk[:, :cut].any() and not gv[:, :cut].any()
+        dK[:, lo + cut:(i + 1) * S] += gk[:, cut:].float()
+        dV[:, lo + cut:(i + 1) * S] += gv[:, cut:].float()
+        if i in (0, 1, L // S - 1):
+            # this segment's term against the oracle: the loss of segment i alone, whole sequence up to its end
+            hi = (i + 1) * S
+            dOw = np.zeros_like(dOf[:, :hi])
+            dOw[:, sl] = dOf[:, sl]
+            rq, rk, rv = oracle.bwd(Qf[:, :hi], Kf[:, :hi], Vf[:, :hi], dOw, S, T, mask)
+            assert not rk[:, :lo + cut].any()          # nothing older than the tail receives gradient
+            assert_grads_close((gq, gk[:, cut:], gv[:, cut:]), (rq[:, sl], rk[:, lo + cut:], rv[:, lo + cut:]), "segment %d" % i)
+    pf.close()
+    O1, LSE1 = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    ref = oracle.bwd(Qf, Kf, Vf, dOf, S, T, mask)
+    assert_grads_close((dQ, dK, dV), ref, "sum over segments")
