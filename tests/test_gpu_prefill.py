@@ -126,3 +126,25 @@ def test_streamed_backward_sums_to_the_one_shot_backward(B, L, Hq, Hkv, d, S, T,
     O1, LSE1 = sa.seg_attn_fwd(Q, K, V, S, T, mask)
     ref = oracle.bwd(Qf, Kf, Vf, dOf, S, T, mask)
     assert_grads_close((dQ, dK, dV), ref, "sum over segments")
+
+
+def test_streamed_backward_needs_a_stepped_segment_and_a_workspace():
+    pf = sa.Prefill(1, 128, 64, 2, 1, 128, 256, [0])
+    q = torch.zeros(1, 128, 2, 128, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(1, 2, 128, dtype=torch.float32, device="cuda")
+    with pytest.raises(sa.SegAttnError):
+        pf.step_bwd(q, q, lse, q)            # nothing stepped yet
+    k = torch.zeros(1, 128, 1, 128, dtype=torch.bfloat16, device="cuda")
+    o, lse = pf.step(q, k, k)
+    pf._bwd_ws = torch.empty(256, dtype=torch.uint8, device="cuda")   # too small and kept: the call must refuse it
+    need = int(sa.lib().seg_prefill_bwd_workspace_bytes(pf._h))
+    assert need > 256
+    import ctypes
+    st = sa.lib().seg_prefill_step_bwd(pf._h, q.data_ptr(), o.data_ptr(), lse.data_ptr(), q.data_ptr(), q.data_ptr(),
+                                       k.data_ptr(), k.data_ptr(), ctypes.c_void_p(pf._bwd_ws.data_ptr()), 256, None)
+    assert st == 5
+    pf._bwd_ws = None
+    dq, dk, dv = pf.step_bwd(q, o, lse, q)   # zero cotangent: zero gradients
+    sa.poll_status()
+    assert not dq.any() and not dk.any() and not dv.any() and dk.shape == (1, 192, 1, 128)
+    pf.close()
