@@ -368,8 +368,8 @@ def run_ours(args, w):
 
 def run_table(args):
     """One JSON line per workload (configurations 1-3 and the 24 points of sweep 5): per-kernel CUDA-event
-    times with inputs resident in HBM, and the throughput over unmasked work they give.  Fills the
-    results table of the benchmark spec; not the benchmark line."""
+    times with inputs resident in HBM, and the throughput over unmasked work they give.  The source of
+    the repository's table of measured results; not the benchmark line."""
     import paper_2605_11744_b200 as sa
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
