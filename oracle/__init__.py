@@ -28,7 +28,7 @@ _lib = None
 class _Cfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "Lq", "Lk", "Hq", "Hkv", "d", "S", "T", "q_pos0", "kv_pos0", "flagged_tail_is_sg", "detach_before")] + \
-               [("scale", ctypes.c_double)]
+               [("scale", ctypes.c_double), ("seg_starts", ctypes.c_void_p), ("n_segs", ctypes.c_int32)]
 
 
 def build(force: bool = False) -> str:
@@ -64,6 +64,16 @@ def _ptr(a):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
 
 
+def _with_starts(cfg, seg_starts):
+    """Attach variable segment starts (kept alive on the struct) or leave the constant length S."""
+    if seg_starts is not None:
+        st = np.ascontiguousarray(np.asarray(seg_starts), dtype=np.int32)
+        cfg._starts = st
+        cfg.seg_starts = st.ctypes.data
+        cfg.n_segs = int(st.size)
+    return cfg
+
+
 def _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg, detach_before=0):
     B, Lq, Hq, d = Q.shape
     Bk, Lk, Hkv, dk = K.shape
@@ -80,10 +90,10 @@ def _mask(head_past_mask, Hkv):
     return m
 
 
-def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False):
+def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False, seg_starts=None):
     """O ``[B,Lq,Hq,d]`` and natural-log LSE ``[B,Hq,Lq]`` of the scaled scores over visible keys."""
     Q, K, V = _f64(Q), _f64(K), _f64(V)
-    cfg = _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg)
+    cfg = _with_starts(_cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg), seg_starts)
     m = _mask(head_past_mask, cfg.Hkv)
     O = np.empty_like(Q)
     LSE = np.empty((cfg.B, cfg.Hq, cfg.Lq), dtype=np.float64)
@@ -95,11 +105,11 @@ def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, fla
 
 
 def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False,
-        detach_before=0):
+        detach_before=0, seg_starts=None):
     """dQ, dK, dV for the cotangent dO; dK/dV hold only what the queries passed in contribute.  Keys at
     global positions below ``detach_before`` are read forward-only (a window with a detached incoming state)."""
     Q, K, V, dO = _f64(Q), _f64(K), _f64(V), _f64(dO)
-    cfg = _cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg, detach_before)
+    cfg = _with_starts(_cfg(Q, K, S, T, scale, q_pos0, kv_pos0, flagged_tail_is_sg, detach_before), seg_starts)
     m = _mask(head_past_mask, cfg.Hkv)
     dQ, dK, dV = np.empty_like(Q), np.empty_like(K), np.empty_like(V)
     rc = _load().oracle_seg_attn_bwd(ctypes.byref(cfg), _ptr(Q), _ptr(K), _ptr(V), _ptr(dO),
@@ -110,9 +120,9 @@ def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0,
     return dQ, dK, dV
 
 
-def count_pairs(B, L, Hq, Hkv, S, T, head_past_mask=None, flagged_tail_is_sg=False, detach_before=0):
+def count_pairs(B, L, Hq, Hkv, S, T, head_past_mask=None, flagged_tail_is_sg=False, detach_before=0, seg_starts=None):
     """(visible, differentiable) query-key pair counts by enumerating the mask row by row."""
-    cfg = _Cfg(B, L, L, Hq, Hkv, 1, S, T, 0, 0, int(bool(flagged_tail_is_sg)), int(detach_before), 1.0)
+    cfg = _with_starts(_Cfg(B, L, L, Hq, Hkv, 1, S, T, 0, 0, int(bool(flagged_tail_is_sg)), int(detach_before), 1.0), seg_starts)
     m = _mask(head_past_mask, Hkv)
     nv, nd = ctypes.c_int64(), ctypes.c_int64()
     rc = _load().oracle_count_pairs(ctypes.byref(cfg), m.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)),

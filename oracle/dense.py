@@ -17,11 +17,19 @@ from __future__ import annotations
 import numpy as np
 
 
-def masks(Lq, Lk, S, T, flag, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False):
+def masks(Lq, Lk, S, T, flag, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False, seg_starts=None):
     p = (q_pos0 + np.arange(Lq))[:, None]
     j = (kv_pos0 + np.arange(Lk))[None, :]
-    seg0 = (p // S) * S
-    a = np.maximum(0, seg0 - T)
+    if seg_starts is None:
+        seg0 = (p // S) * S
+        a = np.maximum(0, seg0 - T)
+    else:
+        # segments of given lengths: the tail is the last min(T, length) positions of the previous segment
+        st = np.asarray(seg_starts)
+        i = np.searchsorted(st, p, side="right") - 1
+        seg0 = st[i]
+        prev0 = np.where(i > 0, st[np.maximum(i - 1, 0)], 0)
+        a = np.maximum(prev0, seg0 - T)
     causal = j <= p
     cls = int(flag)  # head class: 0 local, 1 past access, 2 own segment only
     lo_vis = {0: a, 1: np.zeros_like(a), 2: seg0}[cls]
@@ -31,7 +39,7 @@ def masks(Lq, Lk, S, T, flag, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False):
     return visible, diff
 
 
-def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0):
+def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, seg_starts=None):
     Q, K, V = (np.asarray(x, dtype=np.float64) for x in (Q, K, V))
     B, Lq, Hq, d = Q.shape
     _, Lk, Hkv, _ = K.shape
@@ -42,7 +50,7 @@ def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0):
     LSE = np.full((B, Hq, Lq), -np.inf)
     for h in range(Hq):
         c = h // g
-        vis, _ = masks(Lq, Lk, S, T, flags[c], q_pos0, kv_pos0)
+        vis, _ = masks(Lq, Lk, S, T, flags[c], q_pos0, kv_pos0, seg_starts=seg_starts)
         for b in range(B):
             s = scale * (Q[b, :, h] @ K[b, :, c].T)
             s = np.where(vis, s, -np.inf)
@@ -54,7 +62,8 @@ def fwd(Q, K, V, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0):
     return O, LSE
 
 
-def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False):
+def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0, flagged_tail_is_sg=False,
+        seg_starts=None):
     Q, K, V, dO = (np.asarray(x, dtype=np.float64) for x in (Q, K, V, dO))
     B, Lq, Hq, d = Q.shape
     _, Lk, Hkv, _ = K.shape
@@ -64,7 +73,7 @@ def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0,
     dQ, dK, dV = np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V)
     for h in range(Hq):
         c = h // g
-        vis, dif = masks(Lq, Lk, S, T, flags[c], q_pos0, kv_pos0, flagged_tail_is_sg)
+        vis, dif = masks(Lq, Lk, S, T, flags[c], q_pos0, kv_pos0, flagged_tail_is_sg, seg_starts)
         for b in range(B):
             s = np.where(vis, scale * (Q[b, :, h] @ K[b, :, c].T), -np.inf)
             m = s.max(axis=1, keepdims=True)

@@ -7,7 +7,9 @@
  *
  * What it computes, in the paper's terms (their T is our L, their M is our T):
  *   - The sequence is cut into non-overlapping segments of constant length S
- *     (Section 3.1 "Setup"; Section 3.5 assumes |x^(i)| = S).
+ *     (Section 3.1 "Setup"; Section 3.5 assumes |x^(i)| = S), or, with seg_starts,
+ *     of the lengths m_i the caller gives (Section 3.1 allows them to differ); the
+ *     carried tail of a segment shorter than T is the whole segment.
  *   - Each head runs standard scaled dot-product attention
  *     softmax(Q K^T * scale + mask) V over the concatenation [prefix ; segment]
  *     where a segment query sees every prefix position and the within-segment
@@ -67,13 +69,19 @@ typedef struct {
     int32_t flagged_tail_is_sg;
     int32_t detach_before;   /* keys at global positions below this are read forward-only; 0: none */
     double scale;
+    const int32_t *seg_starts; /* NULL: constant length S.  Else n_segs ascending segment starts, the   */
+    int32_t n_segs;            /* first 0; segment i = [starts[i], starts[i+1]), the last one open-ended */
 } oracle_cfg;
 
 static int cfg_ok(const oracle_cfg *c)
 {
     if (c->B < 0 || c->Lq < 0 || c->Lk < 0 || c->Hq <= 0 || c->Hkv <= 0 || c->d <= 0) return 0;
     if (c->Hq % c->Hkv) return 0;
-    if (c->S <= 0 || c->T < 0 || c->T > c->S) return 0;
+    if (c->seg_starts) {
+        if (c->n_segs < 1 || c->seg_starts[0] != 0 || c->T < 0) return 0;
+        for (int i = 1; i < c->n_segs; ++i)
+            if (c->seg_starts[i] <= c->seg_starts[i - 1]) return 0;
+    } else if (c->S <= 0 || c->T < 0 || c->T > c->S) return 0;
     if (c->q_pos0 < 0 || c->detach_before < 0) return 0;
     return 1;
 }
@@ -81,14 +89,25 @@ static int cfg_ok(const oracle_cfg *c)
 /* first visible / first differentiable global key position of query position p */
 static void row_bounds(const oracle_cfg *c, int flag, long p, long *lo_vis, long *lo_diff)
 {
-    long i = p / c->S;
-    long a = i * (long)c->S - c->T;
+    long seg0, a;   /* start of p's segment; start of the carried tail of the segment before it */
+    if (c->seg_starts) {
+        /* segments of lengths m_i (Section 3.1): the tail is the last min(T, m_{i-1}) positions of segment i-1 */
+        int i = 0;
+        while (i + 1 < c->n_segs && c->seg_starts[i + 1] <= p) ++i;
+        seg0 = c->seg_starts[i];
+        long prev0 = i > 0 ? c->seg_starts[i - 1] : 0;
+        a = seg0 - c->T;
+        if (a < prev0) a = prev0;
+    } else {
+        seg0 = (p / c->S) * (long)c->S;
+        a = seg0 - c->T;
+    }
     if (a < 0) a = 0;
     if (flag == 2) {             /* own segment only (Appendix C, Eq. "ctx", third case) */
-        *lo_vis = *lo_diff = i * (long)c->S;
+        *lo_vis = *lo_diff = seg0;
     } else {
         *lo_vis = flag ? 0 : a;
-        *lo_diff = (flag && c->flagged_tail_is_sg) ? i * (long)c->S : a;
+        *lo_diff = (flag && c->flagged_tail_is_sg) ? seg0 : a;
     }
     /* the boundary state of a truncated chain is a constant (Eq. "truncated-base"): reads of keys
      * before detach_before carry no gradient into K/V */

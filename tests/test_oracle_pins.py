@@ -105,7 +105,7 @@ def test_own_segment_only_heads_are_block_diagonal_for_any_tail():
     np.testing.assert_allclose(dense.fwd(Q, K, V, S, T, head_past_mask=[2, 0])[0], O, atol=TOL)
 
 
-def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False, detach_before=0):
+def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False, detach_before=0, seg_starts=None):
     """For every segment i and head: context = [sg(older past) if flagged ; tail of segment i-1 ;
     own segment], every prefix position visible and the own segment causal (Appendix C), run
     through library attention; stop-gradient realised with .detach() (Definition 3.2)."""
@@ -120,9 +120,10 @@ def recurrence_autograd(Q, K, V, dO, S, T, flags, flagged_tail_is_sg=False, deta
     outs = torch.zeros(B, L, Hq, d, dtype=torch.float64)
     lses = torch.zeros(B, Hq, L, dtype=torch.float64)
     pieces = []
-    for i in range((L + S - 1) // S):
-        s0, s1 = i * S, min(L, (i + 1) * S)
-        a = max(0, s0 - T)
+    bounds = list(range(0, L, S)) if seg_starts is None else [b for b in seg_starts if b < L]
+    for i, s0 in enumerate(bounds):
+        s1 = bounds[i + 1] if i + 1 < len(bounds) else L
+        a = max(bounds[i - 1] if i > 0 else 0, s0 - T)   # the tail is at most the whole previous segment
         for h in range(Hq):
             c = h // g
             ks, vs = [], []
@@ -215,6 +216,38 @@ def test_windows_with_detached_incoming_state_compose_to_depth_one_truncation():
             a[:, sl] += b
     for a, b in zip(acc, full):
         np.testing.assert_allclose(a, b, atol=TOL)
+
+
+# ---- segments of given lengths m_i (Section 3.1) ----------------------------------------------------
+@pytest.mark.parametrize("L,starts,T,flags,variant", [
+    (96, [0, 20, 50, 51, 80], 8, [0, 1], False),       # a one-token segment, a tail longer than its segment
+    (100, [0, 33, 66], 40, [2, 0], False),              # T larger than every segment: the tail is the whole previous one
+    (90, [0, 10, 30, 60], 7, [1, 1], True),
+    (64, [0], 5, [0, 0], False),                        # one open-ended segment: plain causal
+])
+def test_segments_of_given_lengths_with_autograd(L, starts, T, flags, variant):
+    Q, K, V, dO = rand(2, L, 4, 2, 8)
+    o, lse, gq, gk, gv = recurrence_autograd(Q, K, V, dO, None, T, flags, variant, seg_starts=starts)
+    O, LSE = oracle.fwd(Q, K, V, 1, T, head_past_mask=flags, seg_starts=starts)
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, 1, T, head_past_mask=flags, flagged_tail_is_sg=variant, seg_starts=starts)
+    for a, b in ((O, o), (LSE, lse), (dQ, gq), (dK, gk), (dV, gv)):
+        np.testing.assert_allclose(a, b, atol=TOL)
+    if not variant:
+        d2 = dense.bwd(Q, K, V, dO, 1, T, head_past_mask=flags, seg_starts=starts)
+        for a, b in zip((dQ, dK, dV), d2):
+            np.testing.assert_allclose(a, b, atol=TOL)
+        np.testing.assert_allclose(dense.fwd(Q, K, V, 1, T, head_past_mask=flags, seg_starts=starts)[0], O, atol=TOL)
+
+
+def test_equal_given_lengths_are_the_constant_length_case():
+    L, S, T = 100, 32, 9
+    Q, K, V, dO = rand(1, L, 2, 2, 8)
+    starts = list(range(0, L, S))
+    a = oracle.fwd(Q, K, V, S, T, [0, 1]) + oracle.bwd(Q, K, V, dO, S, T, [0, 1])
+    b = oracle.fwd(Q, K, V, 1, T, [0, 1], seg_starts=starts) + oracle.bwd(Q, K, V, dO, 1, T, [0, 1], seg_starts=starts)
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
+    assert oracle.count_pairs(1, L, 2, 2, S, T, [0, 1]) == oracle.count_pairs(1, L, 2, 2, 1, T, [0, 1], seg_starts=starts)
 
 
 # ---- retrieved prefix: [K_ret ; K_i] -------------------------------------------------------------
