@@ -94,6 +94,12 @@ typedef struct {
     int64_t k_stride[3]; /* element strides of K (and dK) */
     int64_t v_stride[3]; /* element strides of V (and dV) */
     int64_t o_stride[3]; /* element strides of O (and dO) */
+    const int32_t* seg_starts; /* NULL: segments of constant length S.  Else a HOST array of n_segs ascending global
+                                * positions, the first 0: segment i is [seg_starts[i], seg_starts[i+1]) and the last one
+                                * is open-ended (segments of lengths m_i, Section 3.1).  S is then ignored, T may exceed
+                                * a segment's length (the carried tail of a short segment is the whole segment), and the
+                                * streamed prefill driver does not take it.  Read before the call returns. */
+    int32_t n_segs;            /* 1 .. 256 when seg_starts is given */
 } seg_attn_params;
 
 /* Bytes of device scratch a call needs (is_bwd = 0: forward, none today; 1: backward, the

@@ -28,7 +28,8 @@ class Params(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("B", "Lq", "kv_len", "Hq", "Hkv", "d", "S", "T", "q_pos0", "kv_pos0")] + \
                [("sm_scale", ctypes.c_float), ("flags", ctypes.c_int32), ("detach_before", ctypes.c_int32),
                 ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
-                ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3)]
+                ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3),
+                ("seg_starts", ctypes.c_void_p), ("n_segs", ctypes.c_int32)]
 
 
 _lib = None
@@ -101,8 +102,17 @@ FLAG_FLAGGED_TAIL_SG = 1   # SEGATTN_FLAG_FLAGGED_TAIL_SG of the C header
 HEAD_LOCAL, HEAD_PAST, HEAD_OWN = 0, 1, 2   # SEGATTN_HEAD_* of the C header: entries of head_past_mask
 
 
+def set_seg_starts(p: "Params", seg_starts) -> None:
+    """Segments of given lengths: `seg_starts` (ascending, first 0) replaces the constant length S."""
+    if seg_starts is not None:
+        arr = np.ascontiguousarray(np.asarray(seg_starts), dtype=np.int32)
+        p._seg_starts = arr          # keeps the host array alive as long as the parameter block
+        p.seg_starts = arr.ctypes.data
+        p.n_segs = int(arr.size)
+
+
 def params_for(Q, K, V, O, S: int, T: int, sm_scale: Optional[float] = None, q_pos0: int = 0,
-               kv_pos0: int = 0, flagged_tail_is_sg: bool = False, detach_before: int = 0) -> Params:
+               kv_pos0: int = 0, flagged_tail_is_sg: bool = False, detach_before: int = 0, seg_starts=None) -> Params:
     """seg_attn_params for [B, L, H, d] tensors (only shapes and strides are read)."""
     B, Lq, Hq, d = Q.shape
     kv_len, Hkv = K.shape[1], K.shape[2]
@@ -111,6 +121,7 @@ def params_for(Q, K, V, O, S: int, T: int, sm_scale: Optional[float] = None, q_p
     p.S, p.T, p.q_pos0, p.kv_pos0 = S, T, q_pos0, kv_pos0
     p.flags = FLAG_FLAGGED_TAIL_SG if flagged_tail_is_sg else 0
     p.detach_before = detach_before
+    set_seg_starts(p, seg_starts)
     p.sm_scale = float(sm_scale if sm_scale is not None else d ** -0.5)
     p.q_stride, p.k_stride, p.v_stride, p.o_stride = _strides3(Q), _strides3(K), _strides3(V), _strides3(O)
     return p
@@ -136,12 +147,12 @@ def workspace_bytes(p: Params, is_bwd: bool) -> int:
 
 
 def seg_attn_fwd(Q, K, V, S: int, T: int, head_past_mask=None, sm_scale=None, q_pos0=0, kv_pos0=0,
-                 out=None, lse=None, stream=None):
+                 out=None, lse=None, stream=None, seg_starts=None):
     """O [B,Lq,Hq,d] bf16 and LSE [B,Hq,Lq] fp32 (natural log) - one call of the C entry point `seg_attn_fwd`."""
     _need_cuda_bf16(Q, K, V)
     O = torch.empty_like(Q) if out is None else out
     LSE = torch.empty((Q.shape[0], Q.shape[2], Q.shape[1]), dtype=torch.float32, device=Q.device) if lse is None else lse
-    p = params_for(Q, K, V, O, S, T, sm_scale, q_pos0, kv_pos0)
+    p = params_for(Q, K, V, O, S, T, sm_scale, q_pos0, kv_pos0, seg_starts=seg_starts)
     m = _mask_arr(head_past_mask, p.Hkv)
     _check(lib().seg_attn_fwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), m.ctypes.data, _ptr(O), _ptr(LSE),
                               None, 0, _stream(stream)), "seg_attn_fwd")
@@ -150,7 +161,7 @@ def seg_attn_fwd(Q, K, V, S: int, T: int, head_past_mask=None, sm_scale=None, q_
 
 def seg_attn_bwd(Q, K, V, O, LSE, dO, S: int, T: int, head_past_mask=None, sm_scale=None, q_pos0=0, kv_pos0=0,
                  workspace: Optional[torch.Tensor] = None, stream=None, flagged_tail_is_sg: bool = False,
-                 detach_before: int = 0):
+                 detach_before: int = 0, seg_starts=None):
     """dQ, dK, dV (bf16) - one call of the C entry point `seg_attn_bwd`.  `flagged_tail_is_sg` selects the
     reading in which flagged heads read the carried tail forward-only as well; keys at global positions
     below `detach_before` are read forward-only (a window of segments whose incoming state is a constant)."""
@@ -160,7 +171,7 @@ def seg_attn_bwd(Q, K, V, O, LSE, dO, S: int, T: int, head_past_mask=None, sm_sc
     dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
     if dQ.stride() != Q.stride() or dK.stride() != K.stride() or dV.stride() != V.stride():
         raise ValueError("Q, K, V must be dense (non-overlapping) tensors")
-    p = params_for(Q, K, V, O, S, T, sm_scale, q_pos0, kv_pos0, flagged_tail_is_sg, detach_before)
+    p = params_for(Q, K, V, O, S, T, sm_scale, q_pos0, kv_pos0, flagged_tail_is_sg, detach_before, seg_starts)
     m = _mask_arr(head_past_mask, p.Hkv)
     need = workspace_bytes(p, True)
     ws = torch.empty(max(need, 256), dtype=torch.uint8, device=Q.device) if workspace is None else workspace
@@ -339,13 +350,14 @@ def launch_count() -> int:
 
 
 def count_pairs(B, Lq, Hq, Hkv, d, S, T, head_past_mask=None, kv_len=None, q_pos0=0, kv_pos0=0,
-                flagged_tail_is_sg: bool = False, detach_before: int = 0):
+                flagged_tail_is_sg: bool = False, detach_before: int = 0, seg_starts=None):
     """(visible pairs, differentiable pairs, 128x128 forward tiles visited), summed over batch and query heads."""
     p = Params()
     p.B, p.Lq, p.kv_len, p.Hq, p.Hkv, p.d, p.S, p.T = B, Lq, Lq if kv_len is None else kv_len, Hq, Hkv, d, S, T
     p.q_pos0, p.kv_pos0, p.sm_scale = q_pos0, kv_pos0, 1.0
     p.flags = FLAG_FLAGGED_TAIL_SG if flagged_tail_is_sg else 0
     p.detach_before = detach_before
+    set_seg_starts(p, seg_starts)
     m = _mask_arr(head_past_mask, Hkv)
     a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
     _check(lib().seg_attn_count_pairs(ctypes.byref(p), m.ctypes.data, ctypes.byref(a), ctypes.byref(b),

@@ -44,6 +44,9 @@ __host__ __device__ inline uint32_t fdiv(uint32_t n, const FastDiv& f) {
     return (uint32_t)(((unsigned long long)hi + n) >> f.s);
 }
 
+constexpr int kMaxSegs = 256;            // segment starts a call can give (segments of unequal length)
+constexpr long long kPosInf = 0x7fffffff;  // "no end": past every supported position
+
 struct MaskGeom {
     FastDiv fS;  // division by S
     int S, T;
@@ -51,13 +54,56 @@ struct MaskGeom {
     int Lq, kv_len;
     int detach_before;    // keys before this global position are read forward-only (0: none)
     int flagged_tail_sg;  // flagged heads read the carried tail forward-only too (Appendix C, Eq. "ctx", read literally)
+    // Segments of given lengths m_i (Section 3.1) instead of the constant S: n_starts > 0 ascending
+    // starts, the first 0, the last segment open-ended.  The carried tail of a segment shorter than T
+    // is the whole segment.
+    int n_starts;
+    int starts[kMaxSegs];
 };
 
 // p / S for a non-negative position (positions fit 32 bits: q_pos0 + Lq is limited to 2^30)
 __host__ __device__ inline long long seg_of(const MaskGeom& g, long long p) {
     return p <= 0xffffffffLL ? (long long)fdiv((uint32_t)p, g.fS) : p / g.S;
 }
+// index of the given-length segment that holds position p (n_starts > 0)
+__host__ __device__ inline int seg_index(const MaskGeom& g, long long p) {
+    int lo = 0, hi = g.n_starts - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (g.starts[mid] <= p) lo = mid;
+        else hi = mid - 1;
+    }
+    return lo;
+}
+// The given-length forms are kept out of line: they run once per work item, and inlining them into
+// the kernels' per-item code costs the constant-length path registers it needs elsewhere.
+#if defined(__CUDACC__)
+#define SEGATTN_NOINLINE __noinline__
+#else
+#define SEGATTN_NOINLINE
+#endif
+__host__ __device__ SEGATTN_NOINLINE inline long long seg_start_given(const MaskGeom& g, long long p) {
+    return (long long)g.starts[seg_index(g, p)];
+}
+__host__ __device__ SEGATTN_NOINLINE inline long long tail_start_given(const MaskGeom& g, long long p) {
+    const int i = seg_index(g, p);
+    const long long prev0 = i > 0 ? g.starts[i - 1] : 0;
+    const long long a = (long long)g.starts[i] - g.T;
+    return a < prev0 ? prev0 : a;
+}
+// one past the last reader of key position j (before the detached-prefix rule)
+__host__ __device__ SEGATTN_NOINLINE inline long long hi_diff_given(const MaskGeom& g, long long j, bool own_only) {
+    const int i = seg_index(g, j);
+    const long long e = i + 1 < g.n_starts ? g.starts[i + 1] : kPosInf;
+    if (own_only || e == kPosInf || j < e - g.T) return e;
+    return i + 2 < g.n_starts ? g.starts[i + 2] : kPosInf;   // a tail position: the next segment reads it too
+}
+// start of p's segment
+__host__ __device__ inline long long seg_start(const MaskGeom& g, long long p) {
+    return g.n_starts ? seg_start_given(g, p) : seg_of(g, p) * (long long)g.S;
+}
 __host__ __device__ inline long long tail_start(const MaskGeom& g, long long p) {
+    if (g.n_starts) return tail_start_given(g, p);
     long long a = seg_of(g, p) * (long long)g.S - g.T;
     return a < 0 ? 0 : a;
 }
@@ -71,18 +117,19 @@ __host__ __device__ inline bool diff_own_only(const MaskGeom& g, int cls) {
 }
 __host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, int cls) {
     if (cls == kHeadPast) return 0;
-    return cls == kHeadOwn ? seg_of(g, p) * (long long)g.S : tail_start(g, p);
+    return cls == kHeadOwn ? seg_start(g, p) : tail_start(g, p);
 }
 // one past the last query position that differentiably reads key position j of a head of class cls
 __host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, int cls) {
     if (j < g.detach_before) return j;  // no differentiable reader at all
+    if (g.n_starts) return hi_diff_given(g, j, diff_own_only(g, cls));
     long long seg_end = (seg_of(g, j) + 1) * (long long)g.S;
     if (diff_own_only(g, cls)) return seg_end;
     return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
 }
 // first key position query position p reads differentiably
 __host__ __device__ inline long long lo_diff(const MaskGeom& g, long long p, int cls) {
-    const long long lo = diff_own_only(g, cls) ? seg_of(g, p) * (long long)g.S : tail_start(g, p);
+    const long long lo = diff_own_only(g, cls) ? seg_start(g, p) : tail_start(g, p);
     return lo < g.detach_before ? g.detach_before : lo;
 }
 

@@ -79,7 +79,14 @@ bool params_ok(const seg_attn_params* p) {
     if (p->B < 0 || p->Lq < 0 || p->kv_len < 0) return false;
     if (p->Hq <= 0 || p->Hkv <= 0 || p->Hkv > kMaxKvHeads || p->Hq % p->Hkv) return false;
     if (p->d != 64 && p->d != 128) return false;
-    if (p->S < 1 || p->T < 0 || p->T > p->S) return false;
+    if (p->S < 1 || p->T < 0) return false;
+    if (p->seg_starts) {
+        if (p->n_segs < 1 || p->n_segs > kMaxSegs || p->seg_starts[0] != 0) return false;
+        for (int i = 1; i < p->n_segs; ++i)
+            if (p->seg_starts[i] <= p->seg_starts[i - 1]) return false;
+    } else if (p->T > p->S) {
+        return false;
+    }
     if (p->q_pos0 < 0 || p->detach_before < 0) return false;
     if (p->flags & ~SEGATTN_FLAG_FLAGGED_TAIL_SG) return false;
     if (!(p->sm_scale > 0.f) || !std::isfinite(p->sm_scale)) return false;
@@ -159,6 +166,8 @@ MaskGeom geom_of(const seg_attn_params* p) {
     g.kv_len = p->kv_len;
     g.flagged_tail_sg = (p->flags & SEGATTN_FLAG_FLAGGED_TAIL_SG) ? 1 : 0;
     g.detach_before = p->detach_before;
+    g.n_starts = p->seg_starts ? p->n_segs : 0;
+    for (int i = 0; i < kMaxSegs; ++i) g.starts[i] = i < g.n_starts ? p->seg_starts[i] : 0;
     return g;
 }
 

@@ -140,6 +140,22 @@ def test_segment_arithmetic_for_many_segment_lengths(S):
     assert hi[:2] == ref[:2]
 
 
+@pytest.mark.parametrize("starts,T", [([0, 20, 50, 51, 300, 700], 8), ([0, 128, 256, 384], 128), ([0], 5),
+                                      ([0, 33, 66], 40), ([0, 1, 2, 3, 500], 2)])
+def test_pair_counter_with_segments_of_given_lengths(starts, T):
+    for mask in ([0, 1], [2, 0]):
+        for X in (0, 60):
+            nv, nd, _ = sa.count_pairs(2, 900, 4, 2, 128, 1, T, mask, seg_starts=starts, detach_before=X)
+            assert (nv, nd) == oracle.count_pairs(2, 900, 4, 2, 1, T, mask, seg_starts=starts, detach_before=X)
+    # equal lengths are the constant-length case
+    S = 128
+    eq = list(range(0, 900, S))
+    assert sa.count_pairs(1, 900, 2, 2, 128, S, 40, [0, 1]) == sa.count_pairs(1, 900, 2, 2, 128, 1, 40, [0, 1], seg_starts=eq)
+    for bad in ([1, 5], [0, 5, 5], [0, 9, 3], list(range(257))):
+        with pytest.raises(sa.SegAttnError):
+            sa.count_pairs(1, 64, 2, 2, 128, 1, 4, [0, 0], seg_starts=bad)
+
+
 def test_unknown_head_class_is_rejected():
     with pytest.raises(sa.SegAttnError):
         sa.count_pairs(1, 256, 2, 2, 128, 64, 16, [0, 3])

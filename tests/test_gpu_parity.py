@@ -238,6 +238,41 @@ def test_empty_and_degenerate_shapes():
     assert torch.count_nonzero(dQ[:, 128:]) == 0
 
 
+@pytest.mark.parametrize("B,L,Hq,Hkv,d,starts,T,mask,X", [
+    (1, 1024, 4, 2, 128, [0, 200, 456, 457, 800], 100, [0, 1], 0),        # a one-token segment; tails longer than it
+    (2, 700, 6, 3, 128, [0, 128, 256, 384, 512], 128, [2, 1, 0], 300),    # tile-aligned; a detached prefix
+    (1, 900, 2, 2, 64, [0, 33, 66, 500], 300, [0, 0], 0),                 # T longer than the short segments
+    (1, 640, 2, 1, 128, [0], 64, [0], 0),                                 # one open-ended segment: plain causal
+    (1, 1500, 2, 2, 128, [0, 700, 1400], 256, [1, 2], 0),                 # long segments, several tiles each
+])
+@pytest.mark.parametrize("tail_sg", [False, True])
+def test_segments_of_given_lengths(B, L, Hq, Hkv, d, starts, T, mask, X, tail_sg):
+    # segments of lengths m_i instead of the constant S; the carried tail of a short segment is all of it
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=L + T)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, 1, T, mask, seg_starts=starts)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, 1, T, mask, flagged_tail_is_sg=tail_sg, detach_before=X,
+                                 seg_starts=starts)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), 1, T, mask, seg_starts=starts)
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), 1, T, mask, flagged_tail_is_sg=tail_sg, detach_before=X,
+                     seg_starts=starts)
+    assert_fwd_close(O, LSE, Oo, LSEo, "fwd")
+    assert_grads_close((dQ, dK, dV), ref, "bwd")
+
+
+def test_equal_given_lengths_are_the_constant_length_path_to_the_bit():
+    B, L, Hq, Hkv, d, S, T, mask = 1, 1000, 4, 2, 128, 256, 100, [0, 1]
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=11)
+    starts = list(range(0, L, S))
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    O2, LSE2 = sa.seg_attn_fwd(Q, K, V, 1, T, mask, seg_starts=starts)
+    assert torch.equal(O, O2) and torch.equal(LSE, LSE2)
+    g1 = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask)
+    g2 = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, 1, T, mask, seg_starts=starts)
+    assert torch.equal(g1[0], g2[0])
+    assert (g1[1].float() - g2[1].float()).abs().max() <= 2e-2     # the dK/dV pass walks its tiles in another order
+
+
 def _random_case(rng):
     d = int(rng.choice([64, 128]))
     Hkv = int(rng.integers(1, 4))
@@ -251,18 +286,22 @@ def _random_case(rng):
     Lk = max(1, q0 + Lq - k0 - (int(rng.integers(0, 200)) if rng.random() < 0.3 else 0))
     mask = [int(rng.integers(0, 3)) for _ in range(Hkv)]
     X = int(rng.integers(0, q0 + Lq + 1)) if rng.random() < 0.4 else 0
+    starts = None
+    if rng.random() < 0.35:   # segments of given lengths instead of the constant S
+        cuts = np.unique(rng.integers(1, q0 + Lq + 1, size=int(rng.integers(0, 7))))
+        starts = [0] + [int(c) for c in cuts]
     return dict(B=int(rng.integers(1, 3)), Lq=Lq, Lk=Lk, Hq=Hkv * g, Hkv=Hkv, d=d, S=S, T=T, q0=q0, k0=k0, mask=mask,
-                X=X, tail_sg=bool(rng.random() < 0.3))
+                X=X, tail_sg=bool(rng.random() < 0.3), starts=starts)
 
 
 @pytest.mark.parametrize("seed", range(64))
 def test_random_shapes_offsets_classes_and_boundaries(seed):
     # seeded random problems over everything the interface takes at once: ragged sizes, position offsets on
     # both sides (keys starting before position 0 or after the first query), head classes, the paper-literal
-    # flag and a detached prefix
+    # flag, a detached prefix and segments of given lengths
     c = _random_case(np.random.default_rng(1000 + seed))
     Q, K, V, dO = rand_inputs(c["B"], c["Lq"], c["Hq"], c["Hkv"], c["d"], seed=seed, Lk=c["Lk"])
-    kw = dict(q_pos0=c["q0"], kv_pos0=c["k0"])
+    kw = dict(q_pos0=c["q0"], kv_pos0=c["k0"], seg_starts=c["starts"])
     O, LSE = sa.seg_attn_fwd(Q, K, V, c["S"], c["T"], c["mask"], **kw)
     dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, c["S"], c["T"], c["mask"], flagged_tail_is_sg=c["tail_sg"],
                                  detach_before=c["X"], **kw)
