@@ -37,9 +37,9 @@ UNIT = "TFLOP/s"
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on the
 # benchmark workload, taken from the ncu captures summarised under profiles/; None = not captured.
 NCU_TRAFFIC_BYTES = {
-    ("cfg2_gqa16k", "fwd"): 647238656,
-    ("cfg2_gqa16k", "dq"): 922862592,
-    ("cfg2_gqa16k", "dkv"): 799855104,
+    ("cfg2_gqa16k", "fwd"): 646085120,
+    ("cfg2_gqa16k", "dq"): 930338560,
+    ("cfg2_gqa16k", "dkv"): 799682816,
 }
 
 
