@@ -434,6 +434,37 @@ def test_host_buffer_step_in_overlapped_chunks(B):
                 assert torch.equal(outs[k], t.cpu()), k
 
 
+def test_a_training_step_captured_in_a_cuda_graph_replays_on_new_data():
+    # nothing in the entry points synchronises, allocates or depends on host state at run time, so a
+    # forward + backward can be captured once and replayed (the launch-bound small shapes gain from it)
+    B, L, Hq, Hkv, d, S, T, mask = 1, 512, 4, 2, 128, 128, 64, [0, 1]
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=21)
+    O = torch.empty_like(Q)
+    LSE = torch.empty(B, Hq, L, dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(256, B * Hq * L * 4 + 256), dtype=torch.uint8, device="cuda")
+    sa.seg_attn_fwd(Q, K, V, S, T, mask, out=O, lse=LSE)          # warm-up outside the capture (function attributes)
+    sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask, workspace=ws)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            sa.seg_attn_fwd(Q, K, V, S, T, mask, out=O, lse=LSE, stream=stream)
+            grads = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask, workspace=ws, stream=stream)
+    for seed in (22, 23):
+        Q2, K2, V2, dO2 = rand_inputs(B, L, Hq, Hkv, d, seed=seed)
+        for dst, src in ((Q, Q2), (K, K2), (V, V2), (dO, dO2)):
+            dst.copy_(src)
+        graph.replay()
+        torch.cuda.synchronize()
+        sa.poll_status()
+        O_e, LSE_e = sa.seg_attn_fwd(Q2, K2, V2, S, T, mask)
+        g_e = sa.seg_attn_bwd(Q2, K2, V2, O_e, LSE_e, dO2, S, T, mask)
+        assert torch.equal(O, O_e) and torch.equal(LSE, LSE_e)
+        for a, b in zip(grads, g_e):
+            assert torch.equal(a, b)
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
     # a wait on a barrier nothing signals gives up after its limit and sets the status word: no hang, no fault
     sa.poll_status()
