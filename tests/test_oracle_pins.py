@@ -10,6 +10,7 @@ import torch.nn.functional as F
 
 import oracle
 from oracle import dense
+from oracle import retrieval
 
 RNG = np.random.default_rng(7)
 TOL = 1e-10
@@ -299,6 +300,63 @@ def test_retrieved_prefix_is_order_free_and_matches_library_attention():
     np.testing.assert_allclose(gq, q.grad.numpy(), atol=TOL)
     np.testing.assert_allclose(gk, ks.grad.numpy(), atol=TOL)
     np.testing.assert_allclose(gv, vs.grad.numpy(), atol=TOL)
+
+
+# ---- selection step of the retrieval operator (Appendix D): mechanics ------------------------------
+def _select_by_sorting(Q, K, Hkv, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R):
+    """The same steps from fp64 scores and library sorting (valid when no two scores tie)."""
+    B, Lq, Hq, d = Q.shape
+    g, P = Hq // Hkv, K.shape[1]
+    n_w = max(1, (Lq - window) // stride + 1) if Lq >= window else 1
+    spans = [(u * stride, min(Lq, u * stride + window)) for u in range(n_w)] + [(max(0, Lq - tail), Lq)]
+    out = np.zeros((B, Hkv, R), dtype=np.int32)
+    for b in range(B):
+        for c in range(Hkv):
+            summ = np.stack([Q[b, r0:r1, c * g:(c + 1) * g].astype(np.float64).mean(axis=(0, 1)) for r0, r1 in spans])
+            sc = summ @ K[b, :, c].astype(np.float64).T
+            cand = sorted(set(np.argsort(-sc, axis=1)[:, :top_k].ravel().tolist()))
+            anchors = sorted(cand, key=lambda j: -sc[:, j].max())[:n_anchors]
+            chosen = []
+            for a in anchors:
+                for j in range(a - off_lo, a + off_hi + 1):
+                    if 0 <= j < P and j not in chosen and len(chosen) < R:
+                        chosen.append(j)
+            chosen += [j for j in range(P) if j not in chosen][:R - len(chosen)]
+            out[b, c] = sorted(chosen)
+    return out
+
+
+@pytest.mark.parametrize("Lq,window,stride,tail,top_k,n_anchors,off_lo,off_hi,R", [
+    (24, 8, 4, 4, 5, 3, 2, 2, 32),
+    (64, 16, 16, 8, 8, 4, 4, 3, 40),
+    (5, 8, 4, 4, 3, 2, 0, 0, 7),          # fewer rows than one window; windows of one position
+    (32, 8, 8, 32, 6, 6, 10, 10, 16),     # R smaller than the windows: best anchors first
+])
+def test_retrieval_selection_against_sorting_and_its_invariants(Lq, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R):
+    rng = np.random.default_rng(Lq + R)
+    Q = rng.standard_normal((2, Lq, 4, 8)).astype(np.float32)
+    K = rng.standard_normal((2, 300, 2, 8)).astype(np.float32)
+    idx = retrieval.select(Q, K, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R)
+    assert idx.shape == (2, 2, R) and idx.dtype == np.int32
+    assert (np.diff(idx, axis=2) > 0).all() and idx.min() >= 0 and idx.max() < 300     # sorted, distinct, in range
+    np.testing.assert_array_equal(idx, _select_by_sorting(Q, K, 2, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R))
+    sc = retrieval.scores(retrieval.summaries(Q, 2, window, stride, tail), K)
+    ref = np.einsum("bcme,bpce->bcmp", retrieval.summaries(Q, 2, window, stride, tail).astype(np.float64), K.astype(np.float64))
+    assert np.abs(sc - ref).max() < 1e-5
+
+
+def test_retrieval_selection_finds_a_planted_key_and_pads_with_the_earliest():
+    rng = np.random.default_rng(5)
+    Q = rng.standard_normal((1, 16, 2, 8)).astype(np.float32)
+    K = (0.01 * rng.standard_normal((1, 500, 1, 8))).astype(np.float32)
+    tail_mean = Q[0, -4:].mean(axis=(0, 1))
+    K[0, 321, 0] = 50.0 * tail_mean                    # by far the best match of the tail summary
+    idx = retrieval.select(Q, K, 8, 8, 4, 1, 1, 3, 2, 12)[0, 0]
+    assert set(range(318, 324)) <= set(idx.tolist())   # the anchor's window
+    assert idx[:6].tolist() == [0, 1, 2, 3, 4, 5]      # and the earliest positions as padding
+    # ties go to the lower position: all keys equal -> the first positions win everything
+    Kc = np.ones((1, 50, 1, 8), dtype=np.float32)
+    assert retrieval.select(Q, Kc, 8, 8, 4, 3, 2, 0, 1, 6)[0, 0].tolist() == [0, 1, 2, 3, 4, 5]
 
 
 # ---- closed form: zero keys => uniform attention over the visible set ---------------------------
