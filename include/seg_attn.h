@@ -212,6 +212,32 @@ segattn_status seg_attn_gather_context(int32_t B, int32_t Hkv, int32_t d, int32_
                                        const void* K_seg, const void* V_seg, const int64_t seg_stride[3],
                                        const int32_t* idx, void* K_ctx, void* V_ctx, void* stream);
 
+/* ---- Selection step of the top-k retrieval operator (Appendix D): which R pool positions a head
+ * retrieves.  The paper names the steps and states none of the constants, so all are parameters here,
+ * and the tie and overflow rules are this library's (equal scores: lower position first; windows are
+ * added best anchor first until R positions are chosen; a short set is padded with the earliest
+ * positions not yet chosen).  Steps per (batch, KV head): (1) query summaries of the last Lq_last
+ * queries of the previous segment - the mean over each sliding window [u*stride, u*stride + window)
+ * and the mean over the last `tail` rows, averaged over the group's query heads; (2) dot-product
+ * scores of every summary against every pool key; (3) the top_k keys per summary, deduplicated;
+ * (4) the n_anchors candidates of highest score; (5) positions anchor - off_lo .. anchor + off_hi,
+ * padded to exactly R, ascending.  Arithmetic is fp32 with separately rounded products and
+ * sequential sums, so the choice is reproducible bit for bit.  Q_last is bf16, contiguous
+ * [B][Lq_last][Hq][d]; K_pool bf16 with element strides pool_stride (batch, position, head) and P
+ * positions; idx (DEVICE, int32 [B][Hkv][R]) is what seg_attn_gather_context takes.  Limits: at most
+ * 16 summaries, summaries * top_k <= 1024, R <= P, top_k <= P.  `workspace`: DEVICE, 256-byte aligned,
+ * seg_retrieval_workspace_bytes(...) bytes (0 = invalid parameters). */
+typedef struct {
+    int32_t Lq_last, window, stride, tail; /* query summaries */
+    int32_t top_k, n_anchors;              /* candidates per summary; anchors kept */
+    int32_t off_lo, off_hi;                /* window around an anchor */
+    int32_t R;                             /* positions returned per head */
+} seg_retrieval_params;
+size_t seg_retrieval_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t P, const seg_retrieval_params* r);
+segattn_status seg_retrieval_select(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t P, const void* Q_last,
+                                    const void* K_pool, const int64_t pool_stride[3], const seg_retrieval_params* r,
+                                    int32_t* idx, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- Whole training-step call with HOST buffers (pinned or pageable): copies Q, K, V, dO to
  * the device arena, runs forward and backward, copies O, LSE, dQ, dK, dV back, and
  * synchronises `stream` before returning.  Host tensors are contiguous in the layouts

@@ -57,6 +57,10 @@ def lib():
         L.seg_prefill_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.seg_prefill_bwd_workspace_bytes.argtypes = [vp]
         L.seg_prefill_step_bwd.argtypes = [vp, vp, vp, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.seg_retrieval_workspace_bytes.restype = ctypes.c_size_t
+        L.seg_retrieval_workspace_bytes.argtypes = [ctypes.c_int32] * 5 + [vp]
+        L.seg_retrieval_select.argtypes = [ctypes.c_int32] * 5 + [vp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, vp,
+                                                                  ctypes.c_size_t, vp]
         L.seg_prefill_reset.argtypes = [vp]
         L.seg_prefill_destroy.argtypes = [vp]
         L.seg_prefill_destroy.restype = None
@@ -250,6 +254,31 @@ def gather_context(K_pool, V_pool, idx, K_seg, V_seg, stream=None):
                                          _ptr(K_seg), _ptr(V_seg), _strides3(K_seg), _ptr(idx), _ptr(K_ctx),
                                          _ptr(V_ctx), _stream(stream)), "seg_attn_gather_context")
     return K_ctx, V_ctx
+
+
+class RetrievalParams(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("Lq_last", "window", "stride", "tail", "top_k", "n_anchors", "off_lo",
+                                               "off_hi", "R")]
+
+
+def retrieval_select(Q_last, K_pool, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R, stream=None):
+    """idx int32 [B, Hkv, R]: the positions a head retrieves from the pool - the C entry point
+    `seg_retrieval_select`.  Q_last [B, Lq_last, Hq, d] contiguous, K_pool [B, P, Hkv, d]."""
+    _need_cuda_bf16(Q_last, K_pool)
+    if not Q_last.is_contiguous():
+        raise ValueError("Q_last must be contiguous")
+    B, Lq, Hq, d = Q_last.shape
+    P, Hkv = K_pool.shape[1], K_pool.shape[2]
+    r = RetrievalParams(Lq, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R)
+    need = int(lib().seg_retrieval_workspace_bytes(B, Hq, Hkv, d, P, ctypes.byref(r)))
+    if need == 0:
+        raise SegAttnError(1, "seg_retrieval_workspace_bytes")
+    ws = torch.empty(need, dtype=torch.uint8, device=Q_last.device)
+    idx = torch.empty((B, Hkv, R), dtype=torch.int32, device=Q_last.device)
+    _check(lib().seg_retrieval_select(B, Hq, Hkv, d, P, _ptr(Q_last), _ptr(K_pool), _strides3(K_pool), ctypes.byref(r),
+                                      _ptr(idx), ctypes.c_void_p(ws.data_ptr()), ws.numel(), _stream(stream)),
+           "seg_retrieval_select")
+    return idx
 
 
 def profile_kernels(Q, K, V, dO, S: int, T: int, head_past_mask=None, sm_scale=None, iters: int = 5, stream=None):

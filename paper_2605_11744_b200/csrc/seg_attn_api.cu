@@ -16,6 +16,7 @@
 #include "fwd_kernel.cuh"
 #include "mask.cuh"
 #include "prefill_kernels.cuh"
+#include "retrieval_kernels.cuh"
 
 using namespace segattn;
 

@@ -5,6 +5,7 @@ import pytest
 import torch
 
 from oracle import dense
+from oracle import retrieval
 import paper_2605_11744_b200 as sa
 from util import assert_fwd_close, assert_grads_close, f64
 
@@ -73,3 +74,53 @@ def test_an_index_out_of_range_is_reported_and_not_read():
     assert torch.equal(Kc[0][keep.cuda()], Kc2[0][keep.cuda()])
     with pytest.raises(sa.SegAttnError):
         sa.gather_context(Kp[:, :, :, :100], Vp[:, :, :, :100], idx, Ks[:, :, :, :100], Vs[:, :, :, :100])   # d = 100
+
+
+@pytest.mark.parametrize("B,P,Hq,Hkv,d,Lq,window,stride,tail,top_k,n_anchors,off_lo,off_hi,R,layout", [
+    (1, 3000, 4, 2, 128, 48, 16, 8, 8, 16, 8, 32, 31, 512, "blhd"),    # R = 512, L_q = 48 as in the paper's range
+    (2, 777, 4, 4, 128, 24, 8, 4, 4, 5, 3, 2, 2, 64, "bhld"),          # nothing aligned; pool stored per head
+    (1, 300, 2, 1, 64, 5, 8, 4, 4, 3, 2, 0, 0, 7, "blhd"),             # fewer rows than a window; d = 64
+    (1, 260, 2, 2, 128, 32, 8, 8, 32, 6, 6, 10, 10, 16, "blhd"),       # R smaller than the windows
+    (1, 64, 2, 2, 128, 60, 4, 4, 4, 60, 4, 1, 1, 64, "blhd"),          # 16 summaries, R = P: everything is retrieved
+])
+def test_retrieval_selection_is_bit_exact(B, P, Hq, Hkv, d, Lq, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R, layout):
+    g = torch.Generator().manual_seed(P + R)
+    mk = lambda *s: torch.randn(*s, generator=g).bfloat16().cuda()
+    Q_last = mk(B, Lq, Hq, d)
+    Kp = mk(B, P, Hkv, d) if layout == "blhd" else mk(B, Hkv, P, d).permute(0, 2, 1, 3)
+    idx = sa.retrieval_select(Q_last, Kp, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R)
+    sa.poll_status()
+    ref = retrieval.select(Q_last.float().cpu().numpy(), Kp.float().cpu().numpy(), window, stride, tail, top_k, n_anchors,
+                           off_lo, off_hi, R)
+    assert np.array_equal(idx.cpu().numpy(), ref)
+
+
+def test_retrieve_gather_attend_end_to_end():
+    # the long-range channel of one segment: select R positions from the pool, gather them, attend over
+    # [retrieved ; own segment]; every stage against its oracle
+    B, P, Hq, Hkv, d, S, R = 1, 2048, 4, 2, 128, 256, 512
+    Kp, Vp, _, Ks, Vs, Q, dO = make(B, P, Hq, Hkv, d, 8, S, seed=77)
+    Q_prev = torch.randn(B, 48, Hq, d, generator=torch.Generator().manual_seed(78)).bfloat16().cuda()
+    idx = sa.retrieval_select(Q_prev, Kp, 16, 8, 8, 16, 8, 32, 31, R)
+    ref_idx = retrieval.select(Q_prev.float().cpu().numpy(), Kp.float().cpu().numpy(), 16, 8, 8, 16, 8, 32, 31, R)
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    Kc, Vc = sa.gather_context(Kp, Vp, idx, Ks, Vs)
+    O, LSE = sa.seg_attn_fwd(Q, Kc, Vc, R + S, 0, [0] * Hkv, q_pos0=R, kv_pos0=0)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, Kc, Vc, O, LSE, dO, R + S, 0, [0] * Hkv, q_pos0=R, kv_pos0=0, detach_before=R)
+    sa.poll_status()
+    Oo, LSEo, gq, gk, gv = dense.retrieved_attention(f64(Q), f64(Kp), f64(Vp), ref_idx, f64(Ks), f64(Vs), f64(dO))
+    assert_fwd_close(O, LSE, Oo, LSEo, "end to end")
+    assert_grads_close((dQ, dK[:, R:], dV[:, R:]), (gq, gk, gv), "end to end")
+
+
+def test_retrieval_selection_rejects_what_it_cannot_hold():
+    Q_last = torch.zeros(1, 8, 2, 128, dtype=torch.bfloat16, device="cuda")
+    Kp = torch.zeros(1, 100, 1, 128, dtype=torch.bfloat16, device="cuda")
+    for kw in (dict(R=101), dict(top_k=101), dict(top_k=0), dict(off_lo=-1), dict(stride=0)):
+        a = dict(window=8, stride=4, tail=4, top_k=4, n_anchors=2, off_lo=1, off_hi=1, R=16)
+        a.update(kw)
+        with pytest.raises(sa.SegAttnError):
+            sa.retrieval_select(Q_last, Kp, **a)
+    many = torch.zeros(1, 40, 2, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(sa.SegAttnError):       # 41 summaries
+        sa.retrieval_select(many, Kp, 1, 1, 4, 4, 2, 1, 1, 16)
