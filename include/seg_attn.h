@@ -184,7 +184,9 @@ segattn_status seg_prefill_step(seg_prefill_handle* h, const void* Qseg, const v
  * global positions [i*S - T, i*S + S) - the previous segment's carried tail, then the segment itself
  * (rows before position 0 are zero).  Older rows of past-access heads are read forward-only and get
  * none.  The caller adds the first T rows to the previous segment's gradients.  `workspace`: DEVICE,
- * 256-byte aligned, at least seg_prefill_bwd_workspace_bytes(h) bytes. */
+ * 256-byte aligned, at least seg_prefill_bwd_workspace_bytes(h) bytes.  SEGATTN_ERR_INVALID when no segment
+ * has been stepped yet or a pointer is null or misaligned, SEGATTN_ERR_WORKSPACE for the workspace; the state
+ * is not modified. */
 size_t seg_prefill_bwd_workspace_bytes(const seg_prefill_handle* h);
 segattn_status seg_prefill_step_bwd(seg_prefill_handle* h, const void* Qseg, const void* Oseg, const float* LSEseg,
                                     const void* dOseg, void* dQseg, void* dKctx, void* dVctx, void* workspace,
@@ -226,7 +228,9 @@ segattn_status seg_attn_gather_context(int32_t B, int32_t Hkv, int32_t d, int32_
  * [B][Lq_last][Hq][d]; K_pool bf16 with element strides pool_stride (batch, position, head) and P
  * positions; idx (DEVICE, int32 [B][Hkv][R]) is what seg_attn_gather_context takes.  Limits: at most
  * 16 summaries, summaries * top_k <= 1024, R <= P, top_k <= P.  `workspace`: DEVICE, 256-byte aligned,
- * seg_retrieval_workspace_bytes(...) bytes (0 = invalid parameters). */
+ * seg_retrieval_workspace_bytes(...) bytes (0 = invalid parameters).  Returns SEGATTN_ERR_INVALID for
+ * parameters outside these limits or misaligned pointers and SEGATTN_ERR_WORKSPACE for a missing, misaligned
+ * or short workspace, before anything is launched; the workspace's contents are scratch. */
 typedef struct {
     int32_t Lq_last, window, stride, tail; /* query summaries */
     int32_t top_k, n_anchors;              /* candidates per summary; anchors kept */
