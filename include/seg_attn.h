@@ -19,6 +19,9 @@
  * With global positions p (query) and j (key), i = p / S and a_i = max(0, i*S - T):
  *     visible(p, j, c) <=> lo_c(p) <= j <= p,  lo_c(p) = a_i (LOCAL), 0 (PAST), i*S (OWN)
  *     diff(p, j, c)    <=> max(lo_c(p), a_i) <= j <= p   (reads that carry gradient into K/V)
+ * With seg_attn_params.seg_starts the segments have the lengths the caller gives instead of S: i is the
+ * segment that holds p, i*S becomes its start s_i, and a_i = max(s_{i-1}, s_i - T) (the carried tail of a
+ * segment shorter than T is the whole segment).
  * Query head h uses KV head c = h / (Hq / Hkv).
  *
  * Conventions that hold for every entry point unless it says otherwise:
