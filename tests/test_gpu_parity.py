@@ -1,6 +1,8 @@
 """GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
 seeded inputs - element by element on small and mid-size cases, on oracle-computable
 sub-problems at the full benchmark sizes."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -294,7 +296,7 @@ def _random_case(rng):
                 X=X, tail_sg=bool(rng.random() < 0.3), starts=starts)
 
 
-@pytest.mark.parametrize("seed", range(64))
+@pytest.mark.parametrize("seed", range(int(os.environ.get("SEGATTN_FUZZ_SEEDS", "64"))))   # more seeds for a soak run
 def test_random_shapes_offsets_classes_and_boundaries(seed):
     # seeded random problems over everything the interface takes at once: ragged sizes, position offsets on
     # both sides (keys starting before position 0 or after the first query), head classes, the paper-literal
