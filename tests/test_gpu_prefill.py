@@ -148,3 +148,42 @@ def test_streamed_backward_needs_a_stepped_segment_and_a_workspace():
     sa.poll_status()
     assert not dq.any() and not dk.any() and not dv.any() and dk.shape == (1, 192, 1, 128)
     pf.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_streamed_forward_and_backward_on_random_problems(seed):
+    # seeded random segment lengths, tails, head classes and group sizes through the streamed driver:
+    # forward against the oracle, per-segment backward summed against the whole-sequence oracle backward
+    from util import assert_grads_close
+    rng = np.random.default_rng(500 + seed)
+    d = int(rng.choice([64, 128]))
+    Hkv = int(rng.integers(1, 4))
+    g = int(rng.choice([1, 2]))
+    S = int(rng.choice([int(rng.integers(1, 60)), 128, int(rng.integers(60, 300))]))
+    T = int(rng.integers(0, S + 1))
+    n_seg = int(rng.integers(1, 5))
+    B, L, Hq = int(rng.integers(1, 3)), S * n_seg, Hkv * g
+    mask = [int(rng.integers(0, 3)) for _ in range(Hkv)]
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=seed)
+    pf = sa.Prefill(B, S, T, Hq, Hkv, d, L, mask)
+    O = torch.empty_like(Q)
+    LSE = torch.empty(B, Hq, L, dtype=torch.float32, device="cuda")
+    dQ = torch.empty_like(Q)
+    dK = torch.zeros(B, L, Hkv, d, dtype=torch.float32, device="cuda")
+    dV = torch.zeros_like(dK)
+    for i in range(n_seg):
+        sl = slice(i * S, (i + 1) * S)
+        q, do = Q[:, sl].contiguous(), dO[:, sl].contiguous()
+        o, lse = pf.step(q, K[:, sl].contiguous(), V[:, sl].contiguous())
+        gq, gk, gv = pf.step_bwd(q, o, lse, do)
+        O[:, sl], LSE[:, :, sl], dQ[:, sl] = o, lse, gq
+        lo = i * S - T
+        cut = max(0, -lo)
+        dK[:, lo + cut:(i + 1) * S] += gk[:, cut:].float()
+        dV[:, lo + cut:(i + 1) * S] += gv[:, cut:].float()
+    sa.poll_status()
+    pf.close()
+    what = "S=%d T=%d n=%d mask=%r d=%d g=%d" % (S, T, n_seg, mask, d, g)
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, mask)
+    assert_fwd_close(O, LSE, Oo, LSEo, what)
+    assert_grads_close((dQ, dK, dV), oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask), what)
