@@ -124,3 +124,30 @@ def test_retrieval_selection_rejects_what_it_cannot_hold():
     many = torch.zeros(1, 40, 2, 128, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(sa.SegAttnError):       # 41 summaries
         sa.retrieval_select(many, Kp, 1, 1, 4, 4, 2, 1, 1, 16)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_retrieval_selection_on_random_parameters(seed):
+    rng = np.random.default_rng(900 + seed)
+    d = int(rng.choice([64, 128]))
+    Hkv = int(rng.integers(1, 4))
+    Hq = Hkv * int(rng.choice([1, 2, 4]))
+    P = int(rng.integers(20, 1500))
+    Lq = int(rng.integers(1, 70))
+    window = int(rng.integers(1, 20))
+    stride = int(rng.integers(max(1, (Lq + 13) // 14), 24))       # at most 15 windows
+    tail = int(rng.integers(1, 16))
+    n_sum = retrieval.n_summaries(Lq, window, stride)
+    top_k = int(rng.integers(1, min(P, 1024 // n_sum) + 1))
+    R = int(rng.integers(1, min(P, 600) + 1))
+    a = dict(window=window, stride=stride, tail=tail, top_k=top_k, n_anchors=int(rng.integers(1, 12)),
+             off_lo=int(rng.integers(0, 40)), off_hi=int(rng.integers(0, 40)), R=R)
+    g = torch.Generator().manual_seed(seed)
+    # coarse values make equal scores likely: the tie rule is exercised too
+    coarse = seed % 3 == 0
+    mk = lambda *s: (torch.randint(-2, 3, s, generator=g).float() if coarse else torch.randn(*s, generator=g)).bfloat16().cuda()
+    Q_last, Kp = mk(1, Lq, Hq, d), mk(1, P, Hkv, d)
+    idx = sa.retrieval_select(Q_last, Kp, **a)
+    sa.poll_status()
+    ref = retrieval.select(Q_last.float().cpu().numpy(), Kp.float().cpu().numpy(), **a)
+    assert np.array_equal(idx.cpu().numpy(), ref), a
