@@ -22,6 +22,7 @@ struct RetrievalParams {
     float* summ;      // [B][Hkv][n_sum][d]
     float* scores;    // [B][Hkv][n_sum][P]
     unsigned* mark;   // [B][Hkv][P]: bit m = in summary m's top-k, bit 30 = candidate, bit 31 = selected
+    int* picks;       // [B][Hkv][n_sum][top_k]: the top-k picks of each summary, in pick order
     int* idx;         // [B][Hkv][R]
     int B, Hq, Hkv, d, P, Lq_last, window, stride, tail, top_k, n_anchors, off_lo, off_hi, R, n_sum;
 };
@@ -88,11 +89,44 @@ __device__ __forceinline__ void take_better(float& v, int& j, float v2, int j2) 
     }
 }
 
-// steps 3-5: one block per (batch, KV head)
+// step 3: one block per (batch, KV head, summary): top_k block-wide arg-max picks over that summary's
+// scores, written in pick order.  Bit m of mark[] is this block's "taken" flag (set atomically: the
+// blocks of the other summaries set their own bits in the same words).
+__global__ void __launch_bounds__(1024) retrieval_topk_kernel(const RetrievalParams prm) {
+    __shared__ float s_v[32];
+    __shared__ int s_j[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m = blockIdx.x % prm.n_sum;
+    const long long bc = blockIdx.x / prm.n_sum;
+    const float* sc = prm.scores + (bc * prm.n_sum + m) * prm.P;
+    unsigned* mark = prm.mark + bc * prm.P;
+    int* picks = prm.picks + (bc * prm.n_sum + m) * prm.top_k;
+    for (int t = 0; t < prm.top_k; ++t) {
+        float v = -INFINITY;
+        int j = 0x7fffffff;
+        for (int q = tid; q < prm.P; q += 1024)
+            if (!((*reinterpret_cast<volatile unsigned*>(mark + q) >> m) & 1u)) take_better(v, j, sc[q], q);
+        for (int o = 16; o > 0; o >>= 1)
+            take_better(v, j, __shfl_xor_sync(0xffffffffu, v, o), __shfl_xor_sync(0xffffffffu, j, o));
+        if (lane == 0) {
+            s_v[warp] = v;
+            s_j[warp] = j;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < 32; ++w) take_better(v, j, s_v[w], s_j[w]);
+            picks[t] = j == 0x7fffffff ? -1 : j;
+            if (j != 0x7fffffff) atomicOr(mark + j, 1u << m);
+        }
+        __threadfence_block();
+        __syncthreads();
+    }
+}
+
+// steps 3 (deduplication), 4 and 5: one block per (batch, KV head)
 __global__ void __launch_bounds__(256) retrieval_select_kernel(const RetrievalParams prm) {
     __shared__ int s_cand[kMaxCandidates];
     __shared__ float s_cscore[kMaxCandidates];
-    __shared__ float s_v[8];
     __shared__ int s_j[8];
     __shared__ int s_n, s_base;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -100,45 +134,30 @@ __global__ void __launch_bounds__(256) retrieval_select_kernel(const RetrievalPa
     const float* sc = prm.scores + bc * prm.n_sum * prm.P;
     volatile unsigned* mark = prm.mark + bc * prm.P;
     int* idx = prm.idx + bc * prm.R;
-    if (tid == 0) s_n = 0;
-    __syncthreads();
-    // step 3: top-k per summary, one block-wide arg-max per pick
-    for (int m = 0; m < prm.n_sum; ++m) {
-        for (int t = 0; t < prm.top_k; ++t) {
-            float v = -INFINITY;
-            int j = 0x7fffffff;
-            for (int q = tid; q < prm.P; q += 256)
-                if (!((mark[q] >> m) & 1u)) take_better(v, j, sc[(long long)m * prm.P + q], q);
-            for (int o = 16; o > 0; o >>= 1)
-                take_better(v, j, __shfl_xor_sync(0xffffffffu, v, o), __shfl_xor_sync(0xffffffffu, j, o));
-            if (lane == 0) {
-                s_v[warp] = v;
-                s_j[warp] = j;
+    if (tid == 0) {
+        // the candidate set, in the order the picks were made (summary by summary)
+        const int* picks = prm.picks + bc * prm.n_sum * prm.top_k;
+        int n = 0;
+        for (int q = 0; q < prm.n_sum * prm.top_k; ++q) {
+            const int j = picks[q];
+            if (j >= 0 && !(mark[j] & (1u << 30)) && n < kMaxCandidates) {
+                mark[j] = mark[j] | (1u << 30);
+                s_cand[n++] = j;
             }
-            __syncthreads();
-            if (tid == 0) {
-                for (int w = 1; w < 8; ++w) take_better(v, j, s_v[w], s_j[w]);
-                if (j != 0x7fffffff) {
-                    unsigned bits = mark[j] | (1u << m);
-                    if (!(bits & (1u << 30)) && s_n < kMaxCandidates) {
-                        bits |= 1u << 30;
-                        s_cand[s_n++] = j;
-                    }
-                    mark[j] = bits;
-                }
-            }
-            __threadfence_block();
-            __syncthreads();
         }
+        s_n = n;
     }
-    // steps 4 and 5 are a few thousand operations: one thread, in the stated order
+    __syncthreads();
+    // a candidate's score: its best over the summaries
+    for (int q = tid; q < s_n; q += 256) {
+        float best = -INFINITY;
+        for (int m = 0; m < prm.n_sum; ++m) best = fmaxf(best, sc[(long long)m * prm.P + s_cand[q]]);
+        s_cscore[q] = best;
+    }
+    __syncthreads();
+    // steps 4 and 5 are a few thousand operations on shared memory: one thread, in the stated order
     if (tid == 0) {
         const int n = s_n;
-        for (int q = 0; q < n; ++q) {
-            float best = -INFINITY;
-            for (int m = 0; m < prm.n_sum; ++m) best = fmaxf(best, sc[(long long)m * prm.P + s_cand[q]]);
-            s_cscore[q] = best;
-        }
         int n_sel = 0;
         const int n_anchor = prm.n_anchors < n ? prm.n_anchors : n;
         for (int a = 0; a < n_anchor; ++a) {
