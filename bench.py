@@ -65,21 +65,38 @@ def flop_model(w, mask, count_pairs):
     }
 
 
+def config_of(w, mask, pairs_visible, pairs_diff, world):
+    """The `config` object of the JSON line: the same keys and values for both arms."""
+    flops = 4.0 * w.d * pairs_visible
+    if w.backward:
+        flops += 10.0 * w.d * pairs_diff + 6.0 * w.d * (pairs_visible - pairs_diff)
+    return {"workload": w.name, "B": w.B, "L": w.L, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "S": w.S, "T": w.T,
+            "past_frac": w.past_frac, "flagged_kv_heads": [int(i) for i in np.nonzero(mask)[0]],
+            "passes": "fwd+bwd" if w.backward else "fwd", "l2": "inputs larger than L2 (no flush)",
+            "parallelism": "replicas" if world > 1 else "single GPU",
+            "pairs_visible": int(pairs_visible), "pairs_diff": int(pairs_diff), "flops_per_step": flops}
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index):
-        self.gpu_index = gpu_index
+    def __init__(self, cuda_ordinal):
+        # nvidia-smi numbers GPUs physically, CUDA numbers the visible ones: select by UUID so that the
+        # samples come from the GPU that is timed
+        try:
+            self.gpu_id = "GPU-" + str(torch.cuda.get_device_properties(cuda_ordinal).uuid)
+        except Exception:
+            self.gpu_id = str(cuda_ordinal)
         self.proc = None
         self.file = None
 
     def start(self):
         try:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.Q,
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, "--query-gpu=" + self.Q,
                                           "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
@@ -127,7 +144,6 @@ def oracle_sample(w, x, seg_lo=1, n_seg=2):
     flagged and one unflagged KV head with their query heads, the queries of `n_seg` consecutive
     segments against all earlier keys.  Returns (seconds, algorithmic FLOPs of the sample, cores, text)."""
     import oracle
-    from paper_2605_11744_b200 import count_pairs
     g = w.Hq // w.Hkv
     mask = x["mask"]
     picks = []
@@ -146,7 +162,7 @@ def oracle_sample(w, x, seg_lo=1, n_seg=2):
         K = workloads.to_f64(x["K"][b:b + 1, :r1, c:c + 1])
         V = workloads.to_f64(x["V"][b:b + 1, :r1, c:c + 1])
         m = [int(mask[c])]
-        vis, dif, _ = count_pairs(1, r1 - r0, g, 1, w.d, w.S, w.T, m, kv_len=r1, q_pos0=r0)
+        vis, dif = oracle.count_pairs(1, r1 - r0, g, 1, w.S, w.T, m, Lk=r1, q_pos0=r0)
         t0 = time.perf_counter()
         oracle.fwd(Q, K, V, w.S, w.T, m, scale=w.sm_scale, q_pos0=r0)
         flops += 4.0 * w.d * vis
@@ -161,10 +177,13 @@ def oracle_sample(w, x, seg_lo=1, n_seg=2):
 
 
 def run_reference(args, w):
-    """The reference arm: the CPU oracle, as it stands, on a bounded sample per step."""
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample per step.  Nothing of the
+    CUDA library is imported or loaded in this arm."""
     rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     if rank != 0:
         return
+    import oracle
     x = workloads.make_inputs(w)
     times, flops, cores, text = [], 0.0, 1, ""
     for i in range(args.warmup + args.steps):
@@ -173,16 +192,18 @@ def run_reference(args, w):
             times.append(s)
     total = sum(times)
     val = flops * len(times) / total / 1e12
+    vis, dif = oracle.count_pairs(w.B, w.L, w.Hq, w.Hkv, w.S, w.T, x["mask"])
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "L": w.L, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "S": w.S, "T": w.T,
-                   "past_frac": w.past_frac, "note": "fp64 CPU oracle on host cores; each step is the bounded sample"},
+        "config": config_of(w, x["mask"], vis, dif, world),
+        "note": "fp64 CPU oracle on host cores; each step is the bounded sample named in cpu_baseline",
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": text},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
+    assert "paper_2605_11744_b200" not in sys.modules, "the reference arm must not load the CUDA library"
     print(json.dumps(line), flush=True)
 
 
@@ -346,12 +367,7 @@ def run_ours(args, w):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "B": w.B, "L": w.L, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "S": w.S, "T": w.T,
-                       "past_frac": w.past_frac, "flagged_kv_heads": [int(i) for i in np.nonzero(mask)[0]],
-                       "passes": "fwd+bwd" if w.backward else "fwd", "l2": "inputs larger than L2 (no flush)",
-                       "parallelism": "replicas" if world > 1 else "single GPU",
-                       "pairs_visible": fm["pairs_visible"], "pairs_diff": fm["pairs_diff"],
-                       "flops_per_step": flops_step},
+            "config": config_of(w, mask, fm["pairs_visible"], fm["pairs_diff"], world),
             "frac_of_bf16_peak": value / world / peaks["bf16"],
             "frac_of_bf16_sustained": value / world / peaks["bf16_sustained"],
             "roofline": roofline, "cpu_baseline": cpu,

@@ -35,7 +35,15 @@
  *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it; no entry point
  *     synchronises the device except where stated.
  *   - Errors are return codes.  Arguments are validated on the host before anything is
- *     launched; on a non-zero return nothing was enqueued and the outputs are untouched.
+ *     launched: SEGATTN_ERR_INVALID, _UNSUPPORTED_ARCH, _WORKSPACE and _TOO_LARGE mean that nothing
+ *     was enqueued and the outputs are untouched.  SEGATTN_ERR_CUDA can also come from a launch or
+ *     copy in the middle of a call's sequence (a backward is three kernels, the host-buffer step
+ *     and the streamed prefill several launches and copies): what was enqueued before it still
+ *     runs, so treat the outputs, and for the streamed prefill the handle's state, as undefined.
+ *   - The kernels share one device status word per process (see seg_attn_poll_status).  Once a
+ *     kernel has set it - a bounded wait that ran out, an index a kernel refused - later kernels
+ *     give up their waits early too, so outputs enqueued after that are undefined until
+ *     seg_attn_poll_status has been called, which reads and clears the word.
  *   - Base pointers must be 16-byte aligned and every stride a multiple of 8 elements
  *     (tiles are moved by TMA).  d is 64 or 128.  0 <= T <= S.  Any Lq, kv_len >= 0.
  *   - Arithmetic: bf16 inputs, fp32 accumulation on the tensor cores, fp32 softmax
@@ -210,8 +218,8 @@ void seg_prefill_destroy(seg_prefill_handle* h);
  * existing entry points on the context: seg_attn_fwd / seg_attn_bwd with Lq = Lseg, kv_len = R + Lseg,
  * q_pos0 = R, kv_pos0 = 0, S = R + Lseg, T = 0, class 0 heads, and, in the backward,
  * detach_before = R (the retrieved rows are forward-only: Definition 3.2, Lemma B.1); rows
- * [R, R + Lseg) of the dK/dV it returns are the segment's gradients.  Choosing the R positions
- * (the scoring and top-k selection of Appendix D) is not part of this library. */
+ * [R, R + Lseg) of the dK/dV it returns are the segment's gradients.  The R positions come from the
+ * caller or from seg_retrieval_select below. */
 segattn_status seg_attn_gather_context(int32_t B, int32_t Hkv, int32_t d, int32_t R, int32_t Lseg, int32_t pool_len,
                                        const void* K_pool, const void* V_pool, const int64_t pool_stride[3],
                                        const void* K_seg, const void* V_seg, const int64_t seg_stride[3],

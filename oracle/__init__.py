@@ -120,9 +120,13 @@ def bwd(Q, K, V, dO, S, T, head_past_mask=None, scale=None, q_pos0=0, kv_pos0=0,
     return dQ, dK, dV
 
 
-def count_pairs(B, L, Hq, Hkv, S, T, head_past_mask=None, flagged_tail_is_sg=False, detach_before=0, seg_starts=None):
-    """(visible, differentiable) query-key pair counts by enumerating the mask row by row."""
-    cfg = _with_starts(_Cfg(B, L, L, Hq, Hkv, 1, S, T, 0, 0, int(bool(flagged_tail_is_sg)), int(detach_before), 1.0), seg_starts)
+def count_pairs(B, L, Hq, Hkv, S, T, head_past_mask=None, flagged_tail_is_sg=False, detach_before=0, seg_starts=None,
+                Lk=None, q_pos0=0, kv_pos0=0):
+    """(visible, differentiable) query-key pair counts by enumerating the mask row by row.  ``L`` query rows
+    starting at global position ``q_pos0`` against ``Lk`` key rows (default ``L``) starting at ``kv_pos0``."""
+    Lk = L if Lk is None else Lk
+    cfg = _with_starts(_Cfg(B, L, Lk, Hq, Hkv, 1, S, T, q_pos0, kv_pos0, int(bool(flagged_tail_is_sg)), int(detach_before), 1.0),
+                       seg_starts)
     m = _mask(head_past_mask, Hkv)
     nv, nd = ctypes.c_int64(), ctypes.c_int64()
     rc = _load().oracle_count_pairs(ctypes.byref(cfg), m.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)),

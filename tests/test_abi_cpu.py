@@ -91,8 +91,20 @@ def test_no_device_means_an_error_not_a_fallback():
     p = _params()
     m = np.zeros(2, dtype=np.uint8)
     ok = ctypes.c_void_p(4096)
-    st = sa.lib().seg_attn_fwd(ctypes.byref(p), ok, ok, ok, m.ctypes.data, ok, ok, None, 0, None)
+    L = sa.lib()
+    st = L.seg_attn_fwd(ctypes.byref(p), ok, ok, ok, m.ctypes.data, ok, ok, None, 0, None)
     assert st in (2, 3)      # unsupported device / CUDA error: never a silent CPU path
+    # the retrieval entry points refuse the same way, before any launch
+    stride = (ctypes.c_int64 * 3)(256 * 2 * 128, 2 * 128, 128)
+    st = L.seg_attn_gather_context(1, 2, 128, 8, 16, 256, ok, ok, stride, ok, ok, stride, ok, ok, ok, None)
+    assert st in (2, 3)
+    r = sa.binding.RetrievalParams(Lq_last=16, window=8, stride=4, tail=4, top_k=4, n_anchors=2, off_lo=1, off_hi=1, R=16)
+    L.seg_retrieval_workspace_bytes.restype = ctypes.c_size_t
+    need = L.seg_retrieval_workspace_bytes(1, 4, 2, 128, 256, ctypes.byref(r))
+    assert need > 0
+    st = L.seg_retrieval_select(1, 4, 2, 128, 256, ok, ok, stride, ctypes.byref(r), ok, ctypes.c_void_p(1 << 20),
+                                ctypes.c_size_t(need), None)
+    assert st in (2, 3)
 
 
 @pytest.mark.parametrize("B,L,Hq,Hkv,S,T,mask", [

@@ -46,3 +46,19 @@ def test_reference_arm_runs_on_rank_zero_only():
                         "--steps", "1", "--warmup", "0", "--config", "1"], env=env, capture_output=True, text=True,
                        timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_reference_arm_never_loads_the_cuda_library():
+    # the arm's own assertion (the package is not in sys.modules when the line is printed) makes the run fail
+    # otherwise; the line carries the same config keys as the product arm's
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                        "--warmup", "0", "--config", "1"], capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
+    import bench
+    import workloads
+    w = workloads.CONFIGS[0]
+    want = bench.config_of(w, workloads.head_past_mask(w.Hkv, w.past_frac, w.seed), 0, 0, 1)
+    assert sorted(line["config"]) == sorted(want)
+    assert line["config"]["pairs_visible"] == 2887680      # 4 heads x (4*512*513/2 + 3*512*128)

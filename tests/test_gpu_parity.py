@@ -10,8 +10,8 @@ import torch
 import oracle
 import workloads
 import paper_2605_11744_b200 as sa
-from util import (TOL_GRAD, assert_fwd_close, assert_grads_close, f64, group_slices, oracle_rows, oracle_window,
-                  rand_inputs, rel_l2)
+from util import (TOL_GRAD, assert_fwd_close, assert_grads_close, f64, group_slices, oracle_last_rows, oracle_rows,
+                  oracle_window, rand_inputs, rel_l2)
 
 pytestmark = pytest.mark.gpu
 
@@ -362,7 +362,21 @@ def test_invalid_arguments_are_rejected_before_launch():
     assert e.value.status == 5                                      # workspace too small
 
 
-def _full_size_check(w, late_rows=24, seg_lo=1):
+def _check_window(w, ref, b, c, hq, O, LSE, grads, what):
+    rows = ref["rows"]
+    assert_fwd_close(O[b:b + 1, rows, hq], LSE[b:b + 1, hq, rows], ref["O"], ref["LSE"], what)
+    if grads is not None:
+        dQ, dK, dV = grads
+        keys = ref["keys"]
+        assert_grads_close((dQ[b:b + 1, rows, hq], dK[b:b + 1, keys, c:c + 1], dV[b:b + 1, keys, c:c + 1]),
+                           (ref["dQ"], ref["dK"], ref["dV"]), what)
+
+
+def _full_size_check(w, late_rows=24, windows=((1, 2),), last_rows=0):
+    """The benchmark's launch configuration at full size against the oracle on sub-problems it can compute: per
+    KV group (one past-access, one not) the windows of whole segments listed in `windows` as (first segment,
+    number of segments; negative = counted from the end; a pair of pairs = (past-access group, other group)),
+    the last `last_rows` rows with the last key tiles, and rows sampled from the last segment."""
     x = workloads.make_inputs(w, device="cuda")
     O, LSE = sa.seg_attn_fwd(x["Q"], x["K"], x["V"], w.S, w.T, x["mask"], w.sm_scale)
     grads = None
@@ -371,16 +385,20 @@ def _full_size_check(w, late_rows=24, seg_lo=1):
     sa.poll_status()
     g = w.Hq // w.Hkv
     b = w.B - 1
+    n_seg_total = (w.L + w.S - 1) // w.S
     rng = np.random.default_rng(w.seed + 1)
     for c, hq in group_slices(x["mask"], g):
-        ref = oracle_window(x, w, b, c, hq, seg_lo)
-        rows = ref["rows"]
-        assert_fwd_close(O[b:b + 1, rows, hq], LSE[b:b + 1, hq, rows], ref["O"], ref["LSE"], "%s window kv%d" % (w.name, c))
-        if grads is not None:
-            dQ, dK, dV = grads
-            keys = ref["keys"]
-            assert_grads_close((dQ[b:b + 1, rows, hq], dK[b:b + 1, keys, c:c + 1], dV[b:b + 1, keys, c:c + 1]),
-                               (ref["dQ"], ref["dK"], ref["dV"]), "%s window kv%d" % (w.name, c))
+        for win in windows:
+            if isinstance(win[0], tuple):
+                win = win[0] if int(x["mask"][c]) == 1 else win[1]
+            seg_lo, n_seg = win
+            if seg_lo < 0:
+                seg_lo += n_seg_total
+            ref = oracle_window(x, w, b, c, hq, seg_lo, n_seg)
+            _check_window(w, ref, b, c, hq, O, LSE, grads, "%s segments %d..%d kv%d" % (w.name, seg_lo, seg_lo + n_seg - 1, c))
+        if last_rows:
+            ref = oracle_last_rows(x, w, b, c, hq, last_rows)
+            _check_window(w, ref, b, c, hq, O, LSE, grads, "%s last %d rows kv%d" % (w.name, last_rows, c))
         # rows sampled from the last segment, where a flagged head's visible range is longest
         last0 = (w.L - 1) // w.S * w.S
         ps = sorted(set(int(p) for p in rng.integers(last0, w.L, size=late_rows)) | {w.L - 1, last0})
@@ -395,17 +413,27 @@ def _full_size_check(w, late_rows=24, seg_lo=1):
 
 
 def test_configuration_2_full_size_sampled():
-    _full_size_check(workloads.CONFIGS[1])
+    # an early window and the last two segments (every key of which has all its readers inside the window)
+    _full_size_check(workloads.CONFIGS[1], windows=((1, 2), (-2, 2)))
 
 
 def test_configuration_3_full_size_sampled_with_outlier_keys():
-    _full_size_check(workloads.CONFIGS[2], late_rows=12)
+    # late window: the last two segments for the local group, the last segment for the past-access group
+    # (its rows read 32K keys each)
+    _full_size_check(workloads.CONFIGS[2], late_rows=12, windows=((1, 2), ((-1, 1), (-2, 2))))
 
 
 @pytest.mark.parametrize("S,T,frac", [(1024, 256, 0.25), (4096, 4096, 0.0), (16384, 1024, 1.0)])
 def test_configuration_5_sweep_points_sampled(S, T, frac):
     w = workloads.CONFIGS[4].with_(S=S, T=T, past_frac=frac, name="cfg5_S%d_T%d_f%g" % (S, T, frac))
-    _full_size_check(w, late_rows=6, seg_lo=1 if S <= 4096 else 0)
+    _full_size_check(w, late_rows=6, windows=((1 if S <= 4096 else 0, 2),))
+
+
+@pytest.mark.parametrize("w", workloads.sweep(), ids=lambda w: w.name)
+def test_configuration_5_every_sweep_point(w):
+    # all 24 points: the last 136 rows of the sequence (the last key tile and a ragged piece of the one before,
+    # with complete dK/dV) and sampled rows of the last segment
+    _full_size_check(w, late_rows=4, windows=(), last_rows=136)
 
 
 def test_host_buffer_step_matches_device_path():

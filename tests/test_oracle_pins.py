@@ -345,6 +345,45 @@ def test_retrieval_selection_against_sorting_and_its_invariants(Lq, window, stri
     assert np.abs(sc - ref).max() < 1e-5
 
 
+def test_retrieval_summaries_written_out_by_hand():
+    # Appendix D "Query construction": sliding-window means plus the mean of the last rows.  Rows q_r = (r, r^2),
+    # so every expected mean below is worked out by hand, not by the span formula.
+    q = lambda n: np.array([[r, r * r] for r in range(n)], dtype=np.float32).reshape(1, n, 1, 2)
+    # 8 rows, window 4, stride 2, tail 2: windows [0,4) [2,6) [4,8), tail rows 6..7
+    assert retrieval.n_summaries(8, 4, 2) == 4
+    np.testing.assert_array_equal(retrieval.summaries(q(8), 1, 4, 2, 2)[0, 0],
+                                  np.array([[1.5, 3.5], [3.5, 13.5], [5.5, 31.5], [6.5, 42.5]], dtype=np.float32))
+    # 7 rows: a window must lie inside the rows present, so row 6 enters through the tail summary only
+    assert retrieval.n_summaries(7, 4, 2) == 3
+    np.testing.assert_array_equal(retrieval.summaries(q(7), 1, 4, 2, 2)[0, 0],
+                                  np.array([[1.5, 3.5], [3.5, 13.5], [5.5, 30.5]], dtype=np.float32))
+    # fewer rows than one window: a single window over what is there (rows 0..2), tail rows 1..2
+    assert retrieval.n_summaries(3, 4, 2) == 2
+    np.testing.assert_allclose(retrieval.summaries(q(3), 1, 4, 2, 2)[0, 0],
+                               np.array([[1.0, 5.0 / 3.0], [1.5, 2.5]]), rtol=1e-6)
+    # a tail longer than the rows present is all rows; stride = window gives disjoint windows
+    np.testing.assert_array_equal(retrieval.summaries(q(4), 1, 2, 2, 9)[0, 0],
+                                  np.array([[0.5, 0.5], [2.5, 6.5], [1.5, 3.5]], dtype=np.float32))
+    # grouped heads: the mean runs over the group's query heads too.  Head 0 rows (r, r^2), head 1 rows (10 + r, 0)
+    Q = np.zeros((1, 4, 2, 2), dtype=np.float32)
+    Q[0, :, 0] = q(4)[0, :, 0]
+    Q[0, :, 1, 0] = 10 + np.arange(4)
+    np.testing.assert_array_equal(retrieval.summaries(Q, 1, 4, 4, 1)[0, 0],
+                                  np.array([[6.5, 1.75], [8.0, 4.5]], dtype=np.float32))
+    # two KV heads of one query head each keep their rows apart
+    out = retrieval.summaries(Q, 2, 4, 4, 1)
+    np.testing.assert_array_equal(out[0, 0], np.array([[1.5, 3.5], [3.0, 9.0]], dtype=np.float32))
+    np.testing.assert_array_equal(out[0, 1], np.array([[11.5, 0.0], [13.0, 0.0]], dtype=np.float32))
+
+
+def test_retrieval_selection_against_sorting_at_a_pool_of_thousands():
+    rng = np.random.default_rng(77)
+    Q = rng.standard_normal((1, 48, 4, 16)).astype(np.float32)
+    K = rng.standard_normal((1, 3000, 2, 16)).astype(np.float32)
+    args = (16, 8, 8, 6, 5, 7, 8, 96)
+    np.testing.assert_array_equal(retrieval.select(Q, K, *args), _select_by_sorting(Q, K, 2, *args))
+
+
 def test_retrieval_selection_finds_a_planted_key_and_pads_with_the_earliest():
     rng = np.random.default_rng(5)
     Q = rng.standard_normal((1, 16, 2, 8)).astype(np.float32)
@@ -492,6 +531,21 @@ def test_benchmark_pair_counts():
     local = 8 * 2048 * 2049 // 2 + 7 * 2048 * 512
     assert nv == 2 * (24 * local + 8 * (16384 * 16385 // 2)) == 3305635840
     assert nd == 2 * 32 * local
+
+
+@pytest.mark.parametrize("q0,L,k0,Lk", [(10, 9, 4, 15), (0, 20, 0, 20), (14, 5, 0, 19), (21, 7, 30, 4)])
+def test_pair_counts_of_a_window_match_enumeration(q0, L, k0, Lk):
+    # a window of queries at q0 against keys at k0: counted pair by pair from the mask's definition
+    S, T, classes = 7, 3, [0, 1]
+    nv = nd = 0
+    for cls in classes:
+        for p in range(q0, q0 + L):
+            a = max(0, (p // S) * S - T)
+            for j in range(max(k0, 0), k0 + Lk):
+                if j <= p and (j >= a or cls == 1):
+                    nv += 1
+                    nd += j >= a
+    assert oracle.count_pairs(1, L, 2, 2, S, T, classes, Lk=Lk, q_pos0=q0, kv_pos0=k0) == (nv, nd)
 
 
 # ---- the two statements of the definition agree; streamed == one-shot ---------------------------

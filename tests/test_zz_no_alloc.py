@@ -5,8 +5,9 @@ already run every other test; passes alone in a fresh process and after the rest
 import pytest
 import torch
 
+import oracle
 import paper_2605_11744_b200 as sa
-from util import TOL_GRAD, f64, rand_inputs, rel_l2
+from util import TOL_GRAD, assert_grads_close, f64, rand_inputs, rel_l2
 
 pytestmark = pytest.mark.gpu
 
@@ -19,6 +20,8 @@ def _both_ways(B, L, Hq, Hkv, d, S, T, mask, seed):
     outs = tuple(torch.full_like(t, float("nan")) for t in (Q, K, V))
     got = sa.seg_attn_bwd_static(Q, K, V, O, LSE, dO, S, T, mask, out=outs)
     sa.poll_status()
+    # and against the fp64 oracle directly, not only through the other entry point
+    assert_grads_close(got, oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask), "static scratch vs oracle")
     return ref, got
 
 
