@@ -253,6 +253,40 @@ segattn_status seg_retrieval_select(int32_t B, int32_t Hq, int32_t Hkv, int32_t 
                                     const void* K_pool, const int64_t pool_stride[3], const seg_retrieval_params* r,
                                     int32_t* idx, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- RoPE re-indexing for prefix concatenation (Section 3.4, paragraph of that name; Appendix E).  When a
+ * prefix of P key/value rows - the carried tail (P = T) or the retrieved rows (P = R) - is put in front of a
+ * segment of m rows, the prefix keys are rotated with positions 0 .. P-1 and the segment's queries and keys with
+ * positions P .. P+m-1; values are not rotated.  (For the carried tail this equals rotating everything at its
+ * global position, since scores depend on position differences only; for retrieved rows it does not, which is
+ * why the pool must hold keys BEFORE rotation.)  "Standard RoPE" is read as the rotation of the pairs
+ * (x[i], x[i + d/2]), i < d/2, by the angle pos * base^(-2i/d):
+ *     y[i] = x[i] cos a - x[i + d/2] sin a,   y[i + d/2] = x[i] sin a + x[i + d/2] cos a.
+ * The angles' cosines and sines come from a table the caller keeps on the device:
+ *   seg_rope_table_bytes   bytes of a table for positions [0, n_pos) (0: invalid d or n_pos; n_pos <= 2^24);
+ *   seg_rope_table         fills `table` (DEVICE, 16-byte aligned, fp32 [n_pos][d/2][2] = (cos, sin)); the angles are
+ *                          formed and their cosines and sines taken in double precision, then rounded to fp32;
+ *   seg_rope_apply         Y[b][r][h][:] = Rot(pos0 + r) X[b][r][h][:] for bf16 X, Y [B][L][H][d] with the element
+ *                          strides given (batch, row, head; multiples of 8; Y may be X); inverse != 0 applies the
+ *                          transposed rotation, which maps a gradient with respect to the rotated tensor back to one
+ *                          with respect to the unrotated tensor (dQ of the segment, and rows [R, R+m) of dK).
+ *                          Arithmetic fp32, output rounded to bf16.  pos0 + L <= n_pos.
+ *   seg_attn_gather_context_rope   seg_attn_gather_context with the re-indexed rotation applied to the keys while
+ *                          they are copied: K_ctx[b][r][c] = Rot(r) K_pool[b][idx[b][c][r]][c] for r < R,
+ *                          K_ctx[b][R + t][c] = Rot(R + t) K_seg[b][t][c]; V_ctx is the plain copy.  Same arguments,
+ *                          limits and error behaviour as seg_attn_gather_context; R + Lseg <= n_pos.  The segment's
+ *                          queries are rotated by seg_rope_apply with pos0 = R.
+ * All four validate their arguments on the host (SEGATTN_ERR_INVALID) and enqueue one kernel on `stream`. */
+size_t seg_rope_table_bytes(int32_t n_pos, int32_t d);
+segattn_status seg_rope_table(int32_t n_pos, int32_t d, double base, float* table, void* stream);
+segattn_status seg_rope_apply(int32_t B, int32_t L, int32_t H, int32_t d, const void* X, const int64_t x_stride[3],
+                              void* Y, const int64_t y_stride[3], int32_t pos0, int32_t inverse, const float* table,
+                              int32_t n_pos, void* stream);
+segattn_status seg_attn_gather_context_rope(int32_t B, int32_t Hkv, int32_t d, int32_t R, int32_t Lseg, int32_t pool_len,
+                                            const void* K_pool, const void* V_pool, const int64_t pool_stride[3],
+                                            const void* K_seg, const void* V_seg, const int64_t seg_stride[3],
+                                            const int32_t* idx, void* K_ctx, void* V_ctx, const float* table,
+                                            int32_t n_pos, void* stream);
+
 /* ---- Whole training-step call with HOST buffers (pinned or pageable): copies Q, K, V, dO to
  * the device arena, runs forward and backward, copies O, LSE, dQ, dK, dV back, and
  * synchronises `stream` before returning.  Host tensors are contiguous in the layouts

@@ -61,6 +61,14 @@ def lib():
         L.seg_retrieval_workspace_bytes.argtypes = [ctypes.c_int32] * 5 + [vp]
         L.seg_retrieval_select.argtypes = [ctypes.c_int32] * 5 + [vp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, vp,
                                                                   ctypes.c_size_t, vp]
+        i64p = ctypes.POINTER(ctypes.c_int64)
+        L.seg_rope_table_bytes.restype = ctypes.c_size_t
+        L.seg_rope_table_bytes.argtypes = [ctypes.c_int32, ctypes.c_int32]
+        L.seg_rope_table.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_double, vp, vp]
+        L.seg_rope_apply.argtypes = [ctypes.c_int32] * 4 + [vp, i64p, vp, i64p, ctypes.c_int32, ctypes.c_int32, vp,
+                                                            ctypes.c_int32, vp]
+        L.seg_attn_gather_context_rope.argtypes = [ctypes.c_int32] * 6 + [vp, vp, i64p, vp, vp, i64p, vp, vp, vp, vp,
+                                                                          ctypes.c_int32, vp]
         L.seg_prefill_reset.argtypes = [vp]
         L.seg_prefill_destroy.argtypes = [vp]
         L.seg_prefill_destroy.restype = None
@@ -253,6 +261,47 @@ def gather_context(K_pool, V_pool, idx, K_seg, V_seg, stream=None):
     _check(lib().seg_attn_gather_context(B, Hkv, d, R, Lseg, P, _ptr(K_pool), _ptr(V_pool), _strides3(K_pool),
                                          _ptr(K_seg), _ptr(V_seg), _strides3(K_seg), _ptr(idx), _ptr(K_ctx),
                                          _ptr(V_ctx), _stream(stream)), "seg_attn_gather_context")
+    return K_ctx, V_ctx
+
+
+def rope_table(n_pos: int, d: int, base: float = 10000.0, device="cuda", stream=None) -> torch.Tensor:
+    """fp32 [n_pos, d/2, 2] = (cos, sin) of pos * base^(-2i/d) - the C entry point `seg_rope_table`."""
+    need = int(lib().seg_rope_table_bytes(n_pos, d))
+    if need == 0 and n_pos != 0:
+        raise SegAttnError(1, "seg_rope_table_bytes")
+    table = torch.empty((n_pos, d // 2, 2), dtype=torch.float32, device=device)
+    _check(lib().seg_rope_table(n_pos, d, float(base), _ptr(table), _stream(stream)), "seg_rope_table")
+    return table
+
+
+def rope_apply(X, table, pos0: int = 0, inverse: bool = False, out=None, stream=None):
+    """Row r of X [B, L, H, d] rotated by position pos0 + r (back, with inverse) - the C entry point `seg_rope_apply`."""
+    _need_cuda_bf16(X)
+    Y = torch.empty_like(X) if out is None else out
+    B, L, H, d = X.shape
+    _check(lib().seg_rope_apply(B, L, H, d, _ptr(X), _strides3(X), _ptr(Y), _strides3(Y), pos0, int(bool(inverse)),
+                                _ptr(table), table.shape[0], _stream(stream)), "seg_rope_apply")
+    return Y
+
+
+def gather_context_rope(K_pool, V_pool, idx, K_seg, V_seg, table, stream=None):
+    """[retrieved rows ; segment rows] with the keys rotated at their re-indexed positions (retrieved row r at r,
+    segment row t at R + t) and the values copied - the C entry point `seg_attn_gather_context_rope`."""
+    _need_cuda_bf16(K_pool, V_pool, K_seg, V_seg)
+    if idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous():
+        raise ValueError("idx must be a contiguous int32 CUDA tensor")
+    B, P, Hkv, d = K_pool.shape
+    R, Lseg = idx.shape[2], K_seg.shape[1]
+    if idx.shape[:2] != (B, Hkv) or K_seg.shape[0] != B or K_seg.shape[2:] != (Hkv, d):
+        raise ValueError("shapes do not fit")
+    if V_pool.stride() != K_pool.stride() or V_seg.stride() != K_seg.stride():
+        raise ValueError("K and V must share strides")
+    K_ctx = torch.empty((B, R + Lseg, Hkv, d), dtype=torch.bfloat16, device=K_pool.device)
+    V_ctx = torch.empty_like(K_ctx)
+    _check(lib().seg_attn_gather_context_rope(B, Hkv, d, R, Lseg, P, _ptr(K_pool), _ptr(V_pool), _strides3(K_pool),
+                                              _ptr(K_seg), _ptr(V_seg), _strides3(K_seg), _ptr(idx), _ptr(K_ctx),
+                                              _ptr(V_ctx), _ptr(table), table.shape[0], _stream(stream)),
+           "seg_attn_gather_context_rope")
     return K_ctx, V_ctx
 
 

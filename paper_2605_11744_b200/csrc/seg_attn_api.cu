@@ -17,6 +17,7 @@
 #include "mask.cuh"
 #include "prefill_kernels.cuh"
 #include "retrieval_kernels.cuh"
+#include "rope_kernels.cuh"
 
 using namespace segattn;
 
@@ -334,6 +335,7 @@ segattn_status seg_attn_count_pairs(const seg_attn_params* p, const uint8_t* hea
 
 #include "seg_attn_bwd_api.inc"
 #include "seg_attn_prefill_api.inc"
+#include "seg_attn_rope_api.inc"
 
 // ---- Self-test of the bounded waits ------------------------------------------------------------
 namespace {

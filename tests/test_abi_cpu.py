@@ -19,7 +19,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "seg_attn.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(seg_(?:attn|prefill)_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(seg_(?:attn|prefill|retrieval|rope)_[a-z_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():

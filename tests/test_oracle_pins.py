@@ -11,6 +11,7 @@ import torch.nn.functional as F
 import oracle
 from oracle import dense
 from oracle import retrieval
+from oracle import rope
 
 RNG = np.random.default_rng(7)
 TOL = 1e-10
@@ -396,6 +397,82 @@ def test_retrieval_selection_finds_a_planted_key_and_pads_with_the_earliest():
     # ties go to the lower position: all keys equal -> the first positions win everything
     Kc = np.ones((1, 50, 1, 8), dtype=np.float32)
     assert retrieval.select(Q, Kc, 8, 8, 4, 3, 2, 0, 1, 6)[0, 0].tolist() == [0, 1, 2, 3, 4, 5]
+
+
+# ---- RoPE re-indexing for prefix concatenation (Section 3.4, Appendix E) -----------------------------
+def test_rope_is_a_complex_rotation_of_the_half_split_pairs():
+    rng = np.random.default_rng(3)
+    d, base = 16, 10000.0
+    x = rng.standard_normal((2, 9, 3, d))
+    pos = np.array([0, 1, 2, 5, 17, 100, 1000, 4095, 70000])
+    y = rope.rotate(x, pos, base)
+    # z_i = x_i + 1j x_{i+d/2} multiplied by exp(1j pos base^(-2i/d)), written out with numpy's complex type
+    z = x[..., : d // 2] + 1j * x[..., d // 2:]
+    w = np.exp(1j * pos[:, None] * base ** (-2.0 * np.arange(d // 2) / d))[:, None, :]
+    zz = z * w
+    np.testing.assert_allclose(y, np.concatenate([zz.real, zz.imag], axis=-1), atol=1e-12)
+    # the library form x cos + rotate_half(x) sin, with torch
+    t = torch.tensor(x)
+    ang = torch.tensor(pos, dtype=torch.float64)[:, None] * torch.pow(torch.tensor(base, dtype=torch.float64),
+                                                                       -torch.arange(0, d, 2, dtype=torch.float64) / d)
+    emb = torch.cat([ang, ang], dim=-1)[:, None, :]
+    rot_half = torch.cat([-t[..., d // 2:], t[..., : d // 2]], dim=-1)
+    np.testing.assert_allclose(y, (t * emb.cos() + rot_half * emb.sin()).numpy(), atol=1e-12)
+    np.testing.assert_array_equal(y[:, 0], x[:, 0])                                   # position 0: identity
+    np.testing.assert_allclose(np.linalg.norm(y, axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-12)
+    np.testing.assert_allclose(rope.rotate(y, pos, base, inverse=True), x, atol=1e-12)  # the transpose undoes it
+    # the first pair turns by pos radians (frequency 1), the last by pos * base^(-(d-2)/d)
+    e0 = np.zeros((1, 1, 1, d)); e0[..., 0] = 1.0
+    r = rope.rotate(e0, [2.0], base)[0, 0, 0]
+    assert abs(r[0] - np.cos(2.0)) < 1e-15 and abs(r[d // 2] - np.sin(2.0)) < 1e-15
+    el = np.zeros((1, 1, 1, d)); el[..., d // 2 - 1] = 1.0
+    r = rope.rotate(el, [3.0], base)[0, 0, 0]
+    assert abs(r[d - 1] - np.sin(3.0 * base ** (-(d - 2.0) / d))) < 1e-15
+
+
+def test_rope_scores_depend_on_the_position_difference_only():
+    rng = np.random.default_rng(4)
+    q, k = rng.standard_normal((1, 1, 1, 32)), rng.standard_normal((1, 1, 1, 32))
+    for a, b in ((5, 3), (900, 17), (0, 40), (123, 123)):
+        lhs = (rope.rotate(q, [a]) * rope.rotate(k, [b])).sum()
+        rhs = (q * rope.rotate(k, [b - a])).sum()
+        assert abs(lhs - rhs) < 1e-11
+        assert abs(lhs - (rope.rotate(q, [a + 1000]) * rope.rotate(k, [b + 1000])).sum()) < 1e-10
+
+
+def test_reindexed_prefix_of_the_preceding_rows_is_attention_under_global_positions():
+    # Appendix E: re-indexing "is equivalent to treating the prefix as preceding context under standard RoPE".
+    # Retrieve exactly the R rows in front of the segment, in order: positions 0..R-1 and R..R+m-1 differ from
+    # the global ones s-R..s+m-1 by a constant, so the attention must equal library attention over those rows
+    # with every tensor rotated at its global position.
+    rng = np.random.default_rng(6)
+    B, Hq, Hkv, d, s, R, m = 2, 4, 2, 16, 40, 12, 9
+    Q = rng.standard_normal((B, s + m, Hq, d))
+    K = rng.standard_normal((B, s + m, Hkv, d))
+    V = rng.standard_normal((B, s + m, Hkv, d))
+    idx = np.broadcast_to(np.arange(s - R, s, dtype=np.int32), (B, Hkv, R)).copy()
+    Kc, Vc, Qr = rope.reindexed_context(K[:, :s], V[:, :s], idx, K[:, s:], V[:, s:], Q[:, s:])
+    # the attention over the rotated context: prefix rows all visible, the segment causal
+    sc = 1.0 / np.sqrt(d)
+    g = Hq // Hkv
+    vis = np.concatenate([np.ones((m, R), bool), np.tril(np.ones((m, m), bool))], axis=1)
+    pos = np.arange(s - R, s + m)
+    Kg, Qg = rope.rotate(K[:, s - R:], pos), rope.rotate(Q[:, s:], pos[R:])
+    for b in range(B):
+        for h in range(Hq):
+            c = h // g
+            a1 = np.where(vis, sc * Qr[b, :, h] @ Kc[b, :, c].T, -np.inf)
+            a2 = np.where(vis, sc * Qg[b, :, h] @ Kg[b, :, c].T, -np.inf)
+            np.testing.assert_allclose(a1, a2, atol=1e-10)
+            p1 = torch.softmax(torch.tensor(a1), dim=-1).numpy()
+            np.testing.assert_allclose(p1 @ Vc[b, :, c], torch.softmax(torch.tensor(a2), dim=-1).numpy() @ V[b, s - R:, c], atol=1e-10)
+    np.testing.assert_array_equal(Vc[:, R:], V[:, s:])                                  # values are not rotated
+    np.testing.assert_array_equal(Vc[:, :R], V[:, s - R:s])
+    # an arbitrary (non-contiguous, per-head) selection: each retrieved key is rotated by its slot, not its origin
+    idx2 = np.stack([np.stack([np.sort(rng.choice(s, R, replace=False)) for _ in range(Hkv)]) for _ in range(B)]).astype(np.int32)
+    Kc2, _, _ = rope.reindexed_context(K[:, :s], V[:, :s], idx2, K[:, s:], V[:, s:], Q[:, s:])
+    for r in (0, 5, R - 1):
+        np.testing.assert_allclose(Kc2[1, r, 1], rope.rotate(K[1:2, idx2[1, 1, r]:idx2[1, 1, r] + 1, 1:2], [r])[0, 0, 0], atol=1e-12)
 
 
 # ---- closed form: zero keys => uniform attention over the visible set ---------------------------
