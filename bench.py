@@ -244,6 +244,30 @@ def measure_prefill(sa, peaks):
             "tflops": fm["fwd"] / t / 1e12, "frac_of_bf16_peak": fm["fwd"] / t / 1e12 / peaks["bf16"]}
 
 
+OTHER_WORKLOADS = ("cfg3_outlier32k", "cfg5_S1024_T256_f0", "cfg5_S4096_T1024_f0.25", "cfg5_S16384_T4096_f1")
+
+
+def measure_other_workloads(sa, peaks, iters):
+    """The larger forward + backward workloads in the same run: per-kernel CUDA-event times with inputs resident
+    in HBM, and the whole-step throughput over unmasked work they add up to.  Compact: one entry per workload."""
+    by_name = {w.name: w for w in list(workloads.CONFIGS) + workloads.sweep()}
+    out = {}
+    for name in OTHER_WORKLOADS:
+        w = by_name[name]
+        x = workloads.make_inputs(w, device="cuda")
+        fm = flop_model(w, x["mask"], sa.count_pairs)
+        per = sa.profile_kernels(x["Q"], x["K"], x["V"], x["dO"], w.S, w.T, x["mask"], w.sm_scale, iters=iters)
+        sa.poll_status()
+        ms = per["fwd"] + per["rowdot"] + per["dq"] + per["dkv"]
+        tf = (fm["fwd"] + fm["bwd"]) / (ms / 1e3) / 1e12
+        out[name] = {"ms_per_step": round(ms, 3), "tflops": round(tf, 1), "frac_of_bf16_peak": round(tf / peaks["bf16"], 3),
+                     "flops_per_step": fm["fwd"] + fm["bwd"],
+                     "ms": {k: round(per[k], 3) for k in ("fwd", "rowdot", "dq", "dkv")}}
+        del x
+        torch.cuda.empty_cache()
+    return out
+
+
 def max_over_ranks(value, world, device):
     """The slowest rank's figure (every multi-GPU number is the maximum over ranks).  The only
     collective of a multi-GPU run; it is outside the data path."""
@@ -361,6 +385,11 @@ def run_ours(args, w):
         prefill = None
         if not args.no_prefill:
             prefill = measure_prefill(sa, peaks)
+        others = None
+        if not args.no_others and world == 1 and w.name == "cfg2_gqa16k":
+            del Q, K, V, dO, O, LSE, x
+            torch.cuda.empty_cache()
+            others = measure_other_workloads(sa, peaks, iters=3)
         t_step = ms_total / args.steps / 1e3
         value = aggregate_value(flops_step, world, t_step)
         line = {
@@ -373,7 +402,7 @@ def run_ours(args, w):
             "roofline": roofline, "cpu_baseline": cpu,
             "e2e": {"value": aggregate_value(flops_step, world, e2e_s / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-            "gpu_launches": launches, "clocks": clocks, "prefill": prefill,
+            "gpu_launches": launches, "clocks": clocks, "prefill": prefill, "configs": others,
         }
     if world > 1:
         dist.barrier()
@@ -421,6 +450,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="benchmark configuration number (1-5); default 2")
     ap.add_argument("--no-prefill", action="store_true", help="skip the configuration-4 streamed prefill measurement")
+    ap.add_argument("--no-others", action="store_true",
+                    help="skip the per-kernel timings of configuration 3 and three sweep points (the `configs` key)")
     ap.add_argument("--table", action="store_true",
                     help="per-kernel timings of configurations 1-3 and the sweep, one JSON line each (not the benchmark line)")
     args = ap.parse_args()

@@ -108,8 +108,8 @@ typedef struct {
     const int32_t* seg_starts; /* NULL: segments of constant length S.  Else a HOST array of n_segs ascending global
                                 * positions, the first 0: segment i is [seg_starts[i], seg_starts[i+1]) and the last one
                                 * is open-ended (segments of lengths m_i, Section 3.1).  S is then ignored, T may exceed
-                                * a segment's length (the carried tail of a short segment is the whole segment), and the
-                                * streamed prefill driver does not take it.  Read before the call returns. */
+                                * a segment's length (the carried tail of a short segment is the whole segment).  The
+                                * streamed prefill driver takes its lengths step by step instead (seg_prefill_step_len).  Read before the call returns. */
     int32_t n_segs;            /* 1 .. 256 when seg_starts is given */
 } seg_attn_params;
 
@@ -171,8 +171,8 @@ segattn_status seg_attn_bwd_static(const seg_attn_params* p, const void* Q, cons
  * past-only pool of Section 3.4), the others keep only the T-position tail.
  *
  * The caller provides one device buffer for all persistent state.  In `p`, Lq is the
- * segment length fed per step (must equal S), kv_len is the maximum total length the pool
- * must hold, q_pos0/kv_pos0 are ignored, and the Q/O strides describe the per-step
+ * segment length fed per step (must equal S; seg_prefill_step_len feeds shorter ones), kv_len is the
+ * maximum total length the pool must hold, q_pos0/kv_pos0 are ignored, and the Q/O strides describe the per-step
  * Q/O segment tensors [B][S][Hq][d], the K/V strides the per-step K/V segment tensors
  * [B][S][Hkv][d].  The handle itself is a small host object (malloc'd by create, freed by
  * destroy). */
@@ -186,6 +186,15 @@ segattn_status seg_prefill_create(const seg_attn_params* p, const uint8_t* head_
  * those rows), then rolls the tail.  Call once per segment, in order, on one stream. */
 segattn_status seg_prefill_step(seg_prefill_handle* h, const void* Qseg, const void* Kseg, const void* Vseg,
                                 void* Oseg, float* LSEseg, void* stream);
+/* The same for a segment of Lseg rows, 1 <= Lseg <= S: segments of lengths m_i (Section 3.1 lets them differ), and
+ * in particular a shorter last segment.  The segment tensors hold Lseg rows per batch element and are addressed with
+ * the strides given at creation; LSE_seg is [B][Hq][Lseg].  The carried tail of a segment shorter than T is the whole
+ * segment (never more than one segment back), as with seg_attn_params.seg_starts, whose whole-sequence forward this
+ * reproduces row for row.  seg_prefill_step(h, ...) is seg_prefill_step_len(h, S, ...).  seg_prefill_step_bwd takes
+ * constant-length streams only: after a step with Lseg != S, or after any step that followed one, it returns
+ * SEGATTN_ERR_INVALID. */
+segattn_status seg_prefill_step_len(seg_prefill_handle* h, int32_t Lseg, const void* Qseg, const void* Kseg,
+                                    const void* Vseg, void* Oseg, float* LSEseg, void* stream);
 /* Backward of the segment stepped last (the streamed form of training with truncation depth 1: a
  * segment is run forward, its loss is differentiated, and credit stops where the carried state
  * entered - definition of the K-truncated objective with K = 1).  Valid after seg_prefill_step and

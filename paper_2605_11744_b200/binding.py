@@ -54,6 +54,7 @@ def lib():
         L.seg_prefill_state_bytes.argtypes = [pp, u8p]
         L.seg_prefill_create.argtypes = [pp, u8p, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
         L.seg_prefill_step.argtypes = [vp, vp, vp, vp, vp, fp, vp]
+        L.seg_prefill_step_len.argtypes = [vp, ctypes.c_int32, vp, vp, vp, vp, fp, vp]
         L.seg_prefill_bwd_workspace_bytes.restype = ctypes.c_size_t
         L.seg_prefill_bwd_workspace_bytes.argtypes = [vp]
         L.seg_prefill_step_bwd.argtypes = [vp, vp, vp, fp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -368,16 +369,30 @@ class Prefill:
         self._h = h
 
     def step(self, Qseg, Kseg, Vseg, out=None, lse=None, stream=None):
+        """The next segment: [B, Lseg, H, d] tensors with Lseg <= S (a view of a [B, S, H, d] buffer when B > 1, so
+        that batch elements keep the strides given at creation) - `seg_prefill_step` / `seg_prefill_step_len`."""
         _need_cuda_bf16(Qseg, Kseg, Vseg)
         p = self.params
-        if tuple(Qseg.shape) != (p.B, p.S, p.Hq, p.d) or tuple(Kseg.shape) != (p.B, p.S, p.Hkv, p.d) or \
-                Kseg.shape != Vseg.shape or not (Qseg.is_contiguous() and Kseg.is_contiguous() and Vseg.is_contiguous()):
-            raise ValueError("segment tensors must be contiguous [B,S,H,d]")
-        O = torch.empty_like(Qseg) if out is None else out
-        LSE = torch.empty((p.B, p.Hq, p.S), dtype=torch.float32, device=Qseg.device) if lse is None else lse
-        _check(lib().seg_prefill_step(self._h, _ptr(Qseg), _ptr(Kseg), _ptr(Vseg), _ptr(O), _ptr(LSE),
-                                      _stream(stream)), "seg_prefill_step")
-        return O, LSE
+        Lseg = Qseg.shape[1]
+
+        def fits(t, H):
+            return (t.dim() == 4 and t.shape[0] == p.B and t.shape[1] == Lseg and t.shape[2] == H and t.shape[3] == p.d and
+                    t.stride(3) == 1 and t.stride(2) == p.d and t.stride(1) == H * p.d and
+                    (p.B == 1 or t.stride(0) == p.S * H * p.d))
+        if not (1 <= Lseg <= p.S and fits(Qseg, p.Hq) and fits(Kseg, p.Hkv) and fits(Vseg, p.Hkv)):
+            raise ValueError("segment tensors must be [B, Lseg <= S, H, d] with the strides of a contiguous [B, S, H, d]")
+        if out is None:
+            out = torch.empty((p.B, p.S, p.Hq, p.d), dtype=torch.bfloat16, device=Qseg.device)[:, :Lseg]
+        if not fits(out, p.Hq):
+            raise ValueError("out must be laid out like the query segment")
+        LSE = torch.empty((p.B, p.Hq, Lseg), dtype=torch.float32, device=Qseg.device) if lse is None else lse
+        if Lseg == p.S:
+            _check(lib().seg_prefill_step(self._h, _ptr(Qseg), _ptr(Kseg), _ptr(Vseg), _ptr(out), _ptr(LSE),
+                                          _stream(stream)), "seg_prefill_step")
+        else:
+            _check(lib().seg_prefill_step_len(self._h, Lseg, _ptr(Qseg), _ptr(Kseg), _ptr(Vseg), _ptr(out), _ptr(LSE),
+                                              _stream(stream)), "seg_prefill_step_len")
+        return out, LSE
 
     def step_bwd(self, Qseg, Oseg, LSEseg, dOseg, stream=None):
         """Backward of the segment stepped last: dQ [B,S,Hq,d] and dK, dV [B,T+S,Hkv,d] for the key/value rows

@@ -16,6 +16,7 @@ struct PrefillCopyParams {
     uint4* Vwin;
     long long seg_stride[3];  // (batch, position, head) of Kseg/Vseg, in uint4 units
     int B, S, T, Hkv, Lmax, n_flag, n_unflag;
+    int rows;           // rows of the incoming segment (S, or fewer for a shorter segment)
     int d16;            // d * 2 / 16: uint4 per head row
     int pos0;           // first global position of this segment
     uint8_t slot_of_head[64];  // KV head -> slot inside its class (pool slot or window slot)
@@ -24,13 +25,13 @@ struct PrefillCopyParams {
 
 // one thread per 16 bytes of the incoming segment (K and V both)
 __global__ void __launch_bounds__(256) prefill_append_kernel(const PrefillCopyParams prm) {
-    const long long n = (long long)prm.B * prm.S * prm.Hkv * prm.d16;
+    const long long n = (long long)prm.B * prm.rows * prm.Hkv * prm.d16;
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     if (idx >= n) return;
     const int e = (int)(idx % prm.d16);
     const int h = (int)((idx / prm.d16) % prm.Hkv);
-    const int r = (int)((idx / ((long long)prm.d16 * prm.Hkv)) % prm.S);
-    const int b = (int)(idx / ((long long)prm.d16 * prm.Hkv * prm.S));
+    const int r = (int)((idx / ((long long)prm.d16 * prm.Hkv)) % prm.rows);
+    const int b = (int)(idx / ((long long)prm.d16 * prm.Hkv * prm.rows));
     const long long src = b * prm.seg_stride[0] + (long long)r * prm.seg_stride[1] + h * prm.seg_stride[2] + e;
     const uint4 k = prm.Kseg[src], v = prm.Vseg[src];
     const int slot = prm.slot_of_head[h];
@@ -45,16 +46,18 @@ __global__ void __launch_bounds__(256) prefill_append_kernel(const PrefillCopyPa
     }
 }
 
-// window rows [S, S+T) (the last T positions of the segment just processed) -> rows [0, T)
-__global__ void __launch_bounds__(256) prefill_roll_tail_kernel(uint4* Kwin, uint4* Vwin, int n_units, int S, int T,
-                                                                int d16) {
-    const long long per = (long long)T * d16;
+// The carried tail: window rows [src_row, src_row + n_rows) (the last positions of the segment just processed)
+// -> rows [dst_row, dst_row + n_rows), which end at row T where the next segment begins.  The two ranges never
+// overlap (the source starts at row T or later).  `pitch` = T + S rows per (batch, head) unit.
+__global__ void __launch_bounds__(256) prefill_roll_tail_kernel(uint4* Kwin, uint4* Vwin, int n_units, int pitch,
+                                                                int src_row, int dst_row, int n_rows, int d16) {
+    const long long per = (long long)n_rows * d16;
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     if (idx >= per * n_units) return;
     const long long u = idx / per, off = idx % per;
-    const long long base = u * (long long)(T + S) * d16;
-    Kwin[base + off] = Kwin[base + (long long)S * d16 + off];
-    Vwin[base + off] = Vwin[base + (long long)S * d16 + off];
+    const long long base = u * (long long)pitch * d16;
+    Kwin[base + (long long)dst_row * d16 + off] = Kwin[base + (long long)src_row * d16 + off];
+    Vwin[base + (long long)dst_row * d16 + off] = Vwin[base + (long long)src_row * d16 + off];
 }
 
 // Gradients of the streamed backward, from the two per-class scratch tensors ([B][n][T+S][d], slot order)

@@ -187,3 +187,65 @@ def test_streamed_forward_and_backward_on_random_problems(seed):
     Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, mask)
     assert_fwd_close(O, LSE, Oo, LSEo, what)
     assert_grads_close((dQ, dK, dV), oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask), what)
+
+
+def run_streamed_lengths(Q, K, V, S, T, mask, lengths):
+    """Segments of the given lengths (each <= S) through the streamed driver."""
+    B, L, Hq, d = Q.shape
+    pf = sa.Prefill(B, S, T, Hq, K.shape[2], d, L, mask)
+    O = torch.empty_like(Q)
+    LSE = torch.empty(B, Hq, L, dtype=torch.float32, device=Q.device)
+    bufs = [torch.empty(B, S, t.shape[2], d, dtype=torch.bfloat16, device="cuda") for t in (Q, K, V)]
+    s0 = 0
+    for m in lengths:
+        views = []
+        for buf, t in zip(bufs, (Q, K, V)):
+            buf[:, :m] = t[:, s0:s0 + m]
+            views.append(buf[:, :m])
+        o, l = pf.step(*views)
+        O[:, s0:s0 + m] = o
+        LSE[:, :, s0:s0 + m] = l
+        s0 += m
+    assert s0 == L
+    sa.poll_status()
+    pf.close()
+    return O, LSE
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,d,S,T,mask,lengths", [
+    (1, 4, 2, 128, 256, 128, [0, 1], [256, 256, 256, 100]),            # a shorter last segment
+    (2, 4, 2, 128, 256, 128, [0, 1], [256, 128, 256, 128, 256]),       # unequal lengths, everything on tile boundaries
+    (1, 2, 2, 128, 300, 100, [0, 1], [300, 37, 1, 250, 300, 64]),      # nothing aligned; a one-token segment;
+                                                                       # segments shorter than the tail
+    (1, 6, 3, 64, 200, 200, [2, 1, 0], [64, 200, 150, 3, 199]),        # d = 64, all head classes, T = S
+    (1, 2, 1, 128, 128, 0, [0], [128, 5, 128]),                        # no tail
+])
+def test_streamed_segments_of_unequal_lengths(B, Hq, Hkv, d, S, T, mask, lengths):
+    # Section 3.1: segments of lengths m_i.  The streamed driver fed those lengths step by step gives the rows of the
+    # whole-sequence forward over the same segment starts (and the oracle's).
+    L = sum(lengths)
+    starts = [0] + list(np.cumsum(lengths)[:-1])
+    Q, K, V, _ = rand_inputs(B, L, Hq, Hkv, d, seed=L + S)
+    O2, LSE2 = run_streamed_lengths(Q, K, V, S, T, mask, lengths)
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), 1, T, mask, seg_starts=starts)
+    assert_fwd_close(O2, LSE2, Oo, LSEo, "streamed, unequal lengths")
+    O1, LSE1 = sa.seg_attn_fwd(Q, K, V, 1, T, mask, seg_starts=starts)
+    if all(m % 128 == 0 for m in lengths) and T % 128 == 0:
+        assert torch.equal(O1, O2) and torch.equal(LSE1, LSE2)     # same tiles in the same order
+    else:
+        assert (O1.float() - O2.float()).abs().max() <= 2e-2
+
+
+def test_streamed_backward_refuses_unequal_lengths_and_oversized_segments():
+    B, Hq, Hkv, d, S, T = 1, 2, 1, 128, 128, 64
+    Q, K, V, dO = rand_inputs(B, 256, Hq, Hkv, d, seed=4)
+    pf = sa.Prefill(B, S, T, Hq, Hkv, d, 256, [0])
+    o, l = pf.step(Q[:, :100], K[:, :100], V[:, :100])
+    with pytest.raises(sa.SegAttnError):
+        pf.step_bwd(Q[:, :128].contiguous(), Q[:, :128].contiguous(), torch.zeros(B, Hq, S, device="cuda"), dO[:, :128].contiguous())
+    with pytest.raises(ValueError):
+        pf.step(Q[:, :200], K[:, :200], V[:, :200])     # longer than S
+    h = pf._h
+    assert sa.lib().seg_prefill_step_len(h, 0, 4096, 4096, 4096, 4096, 4096, None) == 1
+    assert sa.lib().seg_prefill_step_len(h, S + 1, 4096, 4096, 4096, 4096, 4096, None) == 1
+    pf.close()
