@@ -244,6 +244,32 @@ def measure_prefill(sa, peaks):
             "tflops": fm["fwd"] / t / 1e12, "frac_of_bf16_peak": fm["fwd"] / t / 1e12 / peaks["bf16"]}
 
 
+def measure_retrieval(sa, peaks, P=131072, iters=20):
+    """Selection step of the retrieval operator at a 128K pool, two long-range KV heads (configuration 4's), the
+    constants of the tests (48 last queries, 7 summaries, top 16 each, 8 anchors, R = 512): HBM-bound, one read
+    of the pool keys is the algorithmic traffic."""
+    B, Hq, Hkv, d, R = 1, 8, 2, 128, 512
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    mk = lambda *s: torch.randn(*s, device="cuda", generator=gen).bfloat16()
+    Kp, Ql = mk(B, P, Hkv, d), mk(B, 48, Hq, d)
+    args = (16, 8, 8, 16, 8, 32, 31, R)
+    for _ in range(3):
+        sa.retrieval_select(Ql, Kp, *args)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        sa.retrieval_select(Ql, Kp, *args)
+    e1.record()
+    torch.cuda.synchronize()
+    sa.poll_status()
+    ms = e0.elapsed_time(e1) / iters
+    nbytes = B * Hkv * P * d * 2
+    gbs = nbytes / (ms / 1e3) / 1e9
+    return {"pool_positions": P, "kv_heads": Hkv, "R": R, "ms": ms, "algorithmic_bytes": nbytes, "GBps": gbs,
+            "frac_of_hbm": gbs / peaks["hbm"], "bound": "hbm", "launches_per_call": 4}
+
+
 OTHER_WORKLOADS = ("cfg3_outlier32k", "cfg5_S1024_T256_f0", "cfg5_S4096_T1024_f0.25", "cfg5_S16384_T4096_f1")
 
 
@@ -385,6 +411,7 @@ def run_ours(args, w):
         prefill = None
         if not args.no_prefill:
             prefill = measure_prefill(sa, peaks)
+        retrieval = None if args.no_prefill else measure_retrieval(sa, peaks)
         others = None
         if not args.no_others and world == 1 and w.name == "cfg2_gqa16k":
             del Q, K, V, dO, O, LSE, x
@@ -402,7 +429,7 @@ def run_ours(args, w):
             "roofline": roofline, "cpu_baseline": cpu,
             "e2e": {"value": aggregate_value(flops_step, world, e2e_s / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-            "gpu_launches": launches, "clocks": clocks, "prefill": prefill, "configs": others,
+            "gpu_launches": launches, "clocks": clocks, "prefill": prefill, "retrieval": retrieval, "configs": others,
         }
     if world > 1:
         dist.barrier()

@@ -21,6 +21,14 @@ constexpr int kBwdThreads = 384;
 constexpr int kEwWarp0 = 4;   // first element-wise warp
 constexpr int kEwWarps = 8;
 constexpr float kLog2e = 1.4426950408889634f;
+#ifndef SEGATTN_DKV_POLY_EVERY
+#define SEGATTN_DKV_POLY_EVERY 1
+#endif
+#ifndef SEGATTN_DQ_POLY_EVERY
+#define SEGATTN_DQ_POLY_EVERY 4
+#endif
+constexpr int kDqPolyEvery = SEGATTN_DQ_POLY_EVERY;     // every n-th pair of phase A's exponentials of the dQ pass; 0: none
+constexpr int kDkvPolyEvery = SEGATTN_DKV_POLY_EVERY;   // 1: half of phase A's exponentials by polynomial, 2: a quarter; 0: none
 
 // ------------------------------------------------------------------------------------------
 // D[b][h][r] = sum_e dO[b][r][h][e] * O[b][r][h][e]; one group of D/8 threads per row, 16-byte loads,
@@ -117,43 +125,8 @@ struct DqSmem {
     static constexpr uint32_t kDynamic = kTotal + 1024;
 };
 
-struct DqItem {
-    int b, hq, slot, qt;
-    int cls;  // head class of the item's KV head
-};
-__device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) {
-    const HeadTable& ht = prm.heads;
-    const int per_f = ht.n_flagged * prm.g * prm.B;
-    const int per_u = (ht.n_slots - ht.n_flagged) * prm.g * prm.B;
-    const int n_f = per_f * prm.n_qtiles;
-    DqItem it;
-    // quotient and remainder through the launch-time reciprocals (the operands are small and non-negative)
-    uint32_t q, hb, cls_off, cls_n;
-    FastDiv f_cls;
-    if (idx < n_f) {
-        q = fdiv((uint32_t)idx, prm.f_per_f);
-        hb = (uint32_t)idx - q * (uint32_t)per_f;
-        cls_off = 0;
-        cls_n = (uint32_t)ht.n_flagged;
-        f_cls = prm.f_ncls_f;
-    } else {
-        idx -= n_f;
-        q = fdiv((uint32_t)idx, prm.f_per_u);
-        hb = (uint32_t)idx - q * (uint32_t)per_u;
-        cls_off = (uint32_t)ht.n_flagged;
-        cls_n = (uint32_t)(ht.n_slots - ht.n_flagged);
-        f_cls = prm.f_ncls_u;
-    }
-    it.qt = prm.n_qtiles - 1 - (int)q;
-    const uint32_t t = fdiv(hb, prm.f_g);
-    const uint32_t r = hb - t * (uint32_t)prm.g;
-    const uint32_t bb = fdiv(t, f_cls);
-    it.slot = ht.order[cls_off + (t - bb * cls_n)];
-    it.b = (int)bb;
-    it.hq = ht.logical[it.slot] * prm.g + (int)r;
-    it.cls = ht.flag[it.slot];
-    return it;
-}
+using DqItem = WorkItem;
+__device__ __forceinline__ DqItem dq_decode(const BwdParams& prm, int idx) { return decode_item(prm, idx); }
 
 // first visible key tile and number of visible key tiles of a work item of the dQ pass
 __device__ __forceinline__ void dq_item_tiles(const BwdParams& prm, const DqItem& it, int* t_lo, int* n_tiles) {
@@ -375,9 +348,16 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dq_kernel(const _
                     tmem_wait_ld_dep(sv);
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        float t0, t1;
-                        f32x2_unpack(fma_f32x2(f32x2_bits(sv[i], sv[i + 1]), sl2x2, nlse2), t0, t1);
-                        float p0 = ex2(t0), p1 = ex2(t1);
+                        const uint64_t x01 = fma_f32x2(f32x2_bits(sv[i], sv[i + 1]), sl2x2, nlse2);
+                        float p0, p1;
+                        if (kDqPolyEvery > 0 && (i / 2) % (kDqPolyEvery > 0 ? kDqPolyEvery : 1) == 0) {
+                            ex2_poly_x2(x01, p0, p1);
+                        } else {
+                            float t0, t1;
+                            f32x2_unpack(x01, t0, t1);
+                            p0 = ex2(t0);
+                            p1 = ex2(t1);
+                        }
                         if (MASKED) {
                             const int col = c0 + (int)col_off + c * 32 + i;
                             p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
@@ -565,7 +545,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
     const int n_it = n_qt * prm.g;
 
     if (tid == 0) {
-        for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i == kBarPFull || i == kBarDsFull) ? kEwWarps : 1);
+        for (int i = 0; i < kNumBars; ++i)
+            mbar_init(bar(i), (i == kBarPFull || i == kBarDsFull) ? kEwWarps : 1);
         fence_mbar_init();
         prefetch_tmap(&prm.tq);
         prefetch_tmap(&prm.tk);
@@ -718,9 +699,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) seg_attn_bwd_dkv_kernel(const 
                 for (int e = 0; e < 32; e += 4) {
                     const float4 l4 = *reinterpret_cast<const float4*>(&s_lse[buf][col_off + c * 32 + e]);
                     float t0, t1, t2, t3;
-                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[e], sv[e + 1]), sl2x2, f32x2(-l4.x, -l4.y)), t0, t1);
-                    f32x2_unpack(fma_f32x2(f32x2_bits(sv[e + 2], sv[e + 3]), sl2x2, f32x2(-l4.z, -l4.w)), t2, t3);
-                    float p0 = ex2(t0), p1 = ex2(t1), p2 = ex2(t2), p3 = ex2(t3);
+                    const uint64_t x01 = fma_f32x2(f32x2_bits(sv[e], sv[e + 1]), sl2x2, f32x2(-l4.x, -l4.y));
+                    const uint64_t x23 = fma_f32x2(f32x2_bits(sv[e + 2], sv[e + 3]), sl2x2, f32x2(-l4.z, -l4.w));
+                    float p0, p1, p2, p3;
+                    f32x2_unpack(x01, t0, t1);
+                    p0 = ex2(t0);
+                    p1 = ex2(t1);
+                    if (kDkvPolyEvery > 0 && (e / 4) % (kDkvPolyEvery > 0 ? kDkvPolyEvery : 1) == 0) {
+                        ex2_poly_x2(x23, p2, p3);   // this pair on the FMA pipes: phase A is bound by the exp2 unit
+                    } else {
+                        f32x2_unpack(x23, t2, t3);
+                        p2 = ex2(t2);
+                        p3 = ex2(t3);
+                    }
                     if (MASKED) {
                         const int q = q0 + (int)col_off + c * 32 + e;
                         p0 = (q >= qlo && q <= qhi) ? p0 : 0.f;

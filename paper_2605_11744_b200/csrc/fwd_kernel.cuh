@@ -39,45 +39,8 @@ struct FwdSmem {
     static constexpr uint32_t kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
 };
 
-// Decode a position in the work list into a work item, heaviest first: flagged heads (long
-// visible ranges) before the others, late query tiles before early ones.
-struct FwdItem {
-    int b, hq, slot, qt;
-    int cls;  // head class of the item's KV head
-};
-__device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) {
-    const HeadTable& ht = prm.heads;
-    const int per_f = ht.n_flagged * prm.g * prm.B;
-    const int per_u = (ht.n_slots - ht.n_flagged) * prm.g * prm.B;
-    const int n_f = per_f * prm.n_qtiles;
-    FwdItem it;
-    // quotient and remainder through the launch-time reciprocals (the operands are small and non-negative)
-    uint32_t q, hb, cls_off, cls_n;
-    FastDiv f_cls;
-    if (idx < n_f) {
-        q = fdiv((uint32_t)idx, prm.f_per_f);
-        hb = (uint32_t)idx - q * (uint32_t)per_f;
-        cls_off = 0;
-        cls_n = (uint32_t)ht.n_flagged;
-        f_cls = prm.f_ncls_f;
-    } else {
-        idx -= n_f;
-        q = fdiv((uint32_t)idx, prm.f_per_u);
-        hb = (uint32_t)idx - q * (uint32_t)per_u;
-        cls_off = (uint32_t)ht.n_flagged;
-        cls_n = (uint32_t)(ht.n_slots - ht.n_flagged);
-        f_cls = prm.f_ncls_u;
-    }
-    it.qt = prm.n_qtiles - 1 - (int)q;
-    const uint32_t t = fdiv(hb, prm.f_g);
-    const uint32_t r = hb - t * (uint32_t)prm.g;
-    const uint32_t bb = fdiv(t, f_cls);
-    it.slot = ht.order[cls_off + (t - bb * cls_n)];
-    it.b = (int)bb;
-    it.hq = ht.logical[it.slot] * prm.g + (int)r;
-    it.cls = ht.flag[it.slot];
-    return it;
-}
+using FwdItem = WorkItem;
+__device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) { return decode_item(prm, idx); }
 // first visible key tile and number of visible key tiles of a work item
 __device__ __forceinline__ void fwd_item_tiles(const FwdParams& prm, const FwdItem& it, int* t_lo, int* n_tiles) {
     long long jl_lo, jl_hi;

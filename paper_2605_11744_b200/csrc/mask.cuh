@@ -228,4 +228,48 @@ struct alignas(64) BwdParams {
     HeadTable heads;
 };
 
+// One work item of the persistent forward and dQ kernels: a 128-row query tile of one (batch, query head).
+struct WorkItem {
+    int b, hq, slot, qt;
+    int cls;  // head class of the item's KV head
+};
+#if defined(__CUDACC__)
+// Decode a position in the work list into a work item, heaviest first: past-access heads (long visible
+// ranges) before the others, late query tiles before early ones.  Params is FwdParams or BwdParams.
+template <class Params>
+__device__ __forceinline__ WorkItem decode_item(const Params& prm, int idx) {
+    const HeadTable& ht = prm.heads;
+    const int per_f = ht.n_flagged * prm.g * prm.B;
+    const int per_u = (ht.n_slots - ht.n_flagged) * prm.g * prm.B;
+    const int n_f = per_f * prm.n_qtiles;
+    WorkItem it;
+    // quotient and remainder through the launch-time reciprocals (the operands are small and non-negative)
+    uint32_t q, hb, cls_off, cls_n;
+    FastDiv f_cls;
+    if (idx < n_f) {
+        q = fdiv((uint32_t)idx, prm.f_per_f);
+        hb = (uint32_t)idx - q * (uint32_t)per_f;
+        cls_off = 0;
+        cls_n = (uint32_t)ht.n_flagged;
+        f_cls = prm.f_ncls_f;
+    } else {
+        idx -= n_f;
+        q = fdiv((uint32_t)idx, prm.f_per_u);
+        hb = (uint32_t)idx - q * (uint32_t)per_u;
+        cls_off = (uint32_t)ht.n_flagged;
+        cls_n = (uint32_t)(ht.n_slots - ht.n_flagged);
+        f_cls = prm.f_ncls_u;
+    }
+    it.qt = prm.n_qtiles - 1 - (int)q;
+    const uint32_t t = fdiv(hb, prm.f_g);
+    const uint32_t r = hb - t * (uint32_t)prm.g;
+    const uint32_t bb = fdiv(t, f_cls);
+    it.slot = ht.order[cls_off + (t - bb * cls_n)];
+    it.b = (int)bb;
+    it.hq = ht.logical[it.slot] * prm.g + (int)r;
+    it.cls = ht.flag[it.slot];
+    return it;
+}
+#endif
+
 }  // namespace segattn

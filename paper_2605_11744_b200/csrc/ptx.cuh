@@ -286,6 +286,36 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ uint64_t f32x2_fwd(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f32x2_unpack_fwd(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// 2^x for a pair of arguments on the FMA and integer pipes instead of the exp2 unit: x = n + r with n = round(x),
+// r in [-0.5, 0.5]; 2^r by a cubic (relative error 7.5e-5, well inside the bf16 rounding the result gets), 2^n by
+// adding n to the exponent field.  Arguments are clamped to >= -126 (the result is then ~1e-38, as good as 0);
+// they must be below 128.
+__device__ __forceinline__ void ex2_poly_x2(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    f32x2_unpack_fwd(x2, x0, x1);
+    const uint64_t xc = f32x2_fwd(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const float magic = 12582912.f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    uint64_t t, n, r, q;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(t) : "l"(xc), "l"(f32x2_fwd(magic, magic)));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(n) : "l"(t), "l"(f32x2_fwd(-magic, -magic)));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(n), "l"(f32x2_fwd(-1.f, -1.f)), "l"(xc));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(f32x2_fwd(0.055171654f, 0.055171654f)), "l"(r), "l"(f32x2_fwd(0.24261113f, 0.24261113f)));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(r), "l"(f32x2_fwd(0.69326097f, 0.69326097f)));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(q), "l"(r), "l"(f32x2_fwd(0.99992806f, 0.99992806f)));
+    uint32_t t0, t1, q0, q1;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(t0), "=r"(t1) : "l"(t));
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(q0), "=r"(q1) : "l"(q));
+    p0 = __uint_as_float(q0 + (t0 << 23));
+    p1 = __uint_as_float(q1 + (t1 << 23));
+}
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
