@@ -301,9 +301,11 @@ segattn_status seg_attn_gather_context_rope(int32_t B, int32_t Hkv, int32_t d, i
  * synchronises `stream` before returning.  Host tensors are contiguous in the layouts
  * above (strides in `p` are ignored).  dO_host == NULL runs the forward only (gradient
  * outputs are then ignored).  `arena` is a caller-owned DEVICE buffer of at least
- * seg_attn_host_arena_bytes(p) bytes, 256-byte aligned.  The batch is processed in up to four
- * chunks whose copies in, kernels (on `stream`) and copies out overlap; the two side streams
- * and their events are created on first use per device and kept for the life of the process.
+ * seg_attn_host_arena_bytes(p) bytes, 256-byte aligned.  The work is processed in up to eight
+ * chunks - ranges of batch elements or, for batches smaller than that, ranges of KV heads (with
+ * their query heads) of one batch element, each an independent problem - whose copies in, kernels
+ * (on `stream`) and copies out overlap; the two side streams and their events are created on first
+ * use per device and kept for the life of the process.
  * With pageable host memory the copies do not overlap but the result is the same. */
 size_t seg_attn_host_arena_bytes(const seg_attn_params* p);
 segattn_status seg_attn_step_host(const seg_attn_params* p, const void* Q_host, const void* K_host,

@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     if (!mbar_wait(bar(kBarKEmpty + s), (uint32_t)((gj / NK) & 1) ^ 1, 2)) return false;
                     mbar_expect_tx(bar(kBarKFull + s), SM::kTileBytes);
                     for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                        tma_load_4d(sK(s) + pnl * 16384, &prm.tk, bar(kBarKFull + s), pnl * 64, it.slot, (t_lo + j) * kTile,
+                        tma_load_4d(sK(s) + pnl * 16384, &prm.tk, bar(kBarKFull + s), pnl * 64, it.slot, (t_lo + n - 1 - j) * kTile,
                                     it.b);
                     return true;
                 };
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     if (!mbar_wait(bar(kBarVEmpty + s), (uint32_t)((gj / NV) & 1) ^ 1, 3)) return false;
                     mbar_expect_tx(bar(kBarVFull + s), SM::kTileBytes);
                     for (int pnl = 0; pnl < SM::kPanels; ++pnl)
-                        tma_load_4d(sV(s) + pnl * 16384, &prm.tv, bar(kBarVFull + s), pnl * 64, it.slot, (t_lo + j) * kTile,
+                        tma_load_4d(sV(s) + pnl * 16384, &prm.tv, bar(kBarVFull + s), pnl * 64, it.slot, (t_lo + n - 1 - j) * kTile,
                                     it.b);
                     return true;
                 };
@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             for (int j = 0; j < n_tiles; ++j) {
                 const int gj = g + j;
                 if ((gj & 1) != grp) continue;  // the other group's tile
-                const int c0 = (t_lo + j) * kTile;
+                const int c0 = (t_lo + n_tiles - 1 - j) * kTile;
                 const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
                 ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (int)(gj % 3)), (uint32_t)((gj / 3) & 1), 8));
                 if (!ok) break;

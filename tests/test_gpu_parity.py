@@ -464,6 +464,25 @@ def test_host_buffer_step_in_overlapped_chunks(B):
                 assert torch.equal(outs[k], t.cpu()), k
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,mask", [
+    (1, 8, 8, [0, 1, 2, 0, 1, 0, 0, 1]),     # eight chunks of one KV head each
+    (2, 6, 3, [1, 0, 2]),                    # three head ranges per batch element
+    (1, 10, 5, [0, 0, 1, 0, 2]),             # five ranges of one head, two query heads each
+    (3, 4, 2, [0, 1]),                       # 3 x 2 chunks
+])
+def test_host_buffer_step_in_chunks_of_kv_heads(B, Hq, Hkv, mask):
+    # a batch smaller than the number of chunks is cut along the KV heads: every (batch element, KV head) is an
+    # independent problem, so the results are those of one launch over everything, bit for bit
+    L, d, S, T = 512, 128, 256, 128
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=B + Hkv, device="cpu")
+    outs = sa.seg_attn_step_host(Q, K, V, dO, S, T, mask)
+    Qd, Kd, Vd, dOd = (t.cuda() for t in (Q, K, V, dO))
+    O, LSE = sa.seg_attn_fwd(Qd, Kd, Vd, S, T, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Qd, Kd, Vd, O, LSE, dOd, S, T, mask)
+    for k, t in (("O", O), ("LSE", LSE), ("dQ", dQ), ("dK", dK), ("dV", dV)):
+        assert torch.equal(outs[k], t.cpu()), k
+
+
 def test_a_training_step_captured_in_a_cuda_graph_replays_on_new_data():
     # nothing in the entry points synchronises, allocates or depends on host state at run time, so a
     # forward + backward can be captured once and replayed (the launch-bound small shapes gain from it)
