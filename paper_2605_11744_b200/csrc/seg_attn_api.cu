@@ -45,6 +45,15 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// SEGATTN_LOG=1 in the environment: one line per launch on stderr with the shapes and the schedule's size.
+bool log_on() {
+    static const bool on = [] {
+        const char* v = getenv("SEGATTN_LOG");
+        return v && *v && *v != '0';
+    }();
+    return on;
+}
+
 segattn_status cuda_fail(cudaError_t e) {
     t_last_cuda_error = (int)e;
     return SEGATTN_ERR_CUDA;
@@ -221,6 +230,11 @@ segattn_status launch_fwd(const seg_attn_params* p, const HeadTable& heads, cons
     int n_sm = 0;
     if ((st = sm_count(&n_sm)) != SEGATTN_OK) return st;
     const unsigned grid = (unsigned)(n_items < n_sm ? n_items : n_sm);
+    if (log_on())
+        fprintf(stderr, "[segattn] fwd: B=%d Lq=%d kv_len=%d Hq=%d Hkv=%d d=%d S=%d T=%d q_pos0=%d kv_pos0=%d segs=%d "
+                        "slots=%d past_slots=%d items=%lld grid=%u\n",
+                p->B, p->Lq, p->kv_len, p->Hq, p->Hkv, p->d, p->S, p->T, p->q_pos0, p->kv_pos0, prm.geom.n_starts,
+                heads.n_slots, heads.n_flagged, n_items, grid);
     if (p->d == 128) {
         if ((st = set_smem(seg_attn_fwd_kernel<128>, FwdSmem<128>::kDynamic)) != SEGATTN_OK) return st;
         seg_attn_fwd_kernel<128><<<grid, kFwdThreads, FwdSmem<128>::kDynamic, stream>>>(prm);

@@ -527,3 +527,24 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
     O, LSE = sa.seg_attn_fwd(Q, K, V, 128, 64, [0])
     Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), 128, 64, [0])
     assert_fwd_close(O, LSE, Oo, LSEo, "after a timeout")
+
+
+def test_launch_log_on_request():
+    # SEGATTN_LOG=1: one line per launch on stderr with the shapes and the size of the schedule
+    import subprocess
+    import sys
+    code = ("import torch, paper_2605_11744_b200 as sa\n"
+            "mk = lambda H: torch.zeros(1, 256, H, 128, dtype=torch.bfloat16, device='cuda')\n"
+            "Q, K, V = mk(2), mk(1), mk(1)\n"
+            "O, LSE = sa.seg_attn_fwd(Q, K, V, 128, 64, [1])\n"
+            "sa.seg_attn_bwd(Q, K, V, O, LSE, Q, 128, 64, [1])\n"
+            "sa.poll_status()\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, SEGATTN_LOG="1", PYTHONPATH=root), capture_output=True,
+                       text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    assert "[segattn] fwd: B=1 Lq=256 kv_len=256 Hq=2 Hkv=1 d=128 S=128 T=64" in r.stderr and "items=4 grid=4" in r.stderr
+    assert "[segattn] bwd dQ pass:" in r.stderr and "[segattn] bwd dK/dV pass: key tiles=2" in r.stderr
+    quiet = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, PYTHONPATH=root, SEGATTN_LOG="0"),
+                           capture_output=True, text=True, timeout=300)
+    assert quiet.returncode == 0 and "[segattn]" not in quiet.stderr
