@@ -7,12 +7,13 @@
 // owner, warp 2 = tcgen05 issuer of the score products,
 // warps 4..7 and 8..11 = two softmax groups (thread = query row) that take the key tiles of even
 // and odd index in turn and pass the running row maximum on through shared memory, then share the
-// epilogue; warp 3 idle.
-// TMEM (512 columns): three S buffers at [0,384), used by the key tiles in turn (P, bf16, is written
-// over the first 64 columns of the tile's S buffer), O at [384,384+D).
-// Tensor-core order per key tile j:  PV(j) | S(j+3): the scores of the next tiles are ready before a
-// softmax group finishes its current tile, so both groups work without waiting for the tensor
-// cores, and rings of K and V tiles keep TMA ahead of both.
+// epilogue; warp 3 idle.  The issuing warpgroup gives most of its registers to the softmax groups,
+// whose threads hold a whole row of scores (128 values) in registers.
+// TMEM (512 columns): one S buffer per softmax group at [0,256), one P buffer (bf16) per group at
+// [256,384), O at [384,384+D).  A group reads its tile's scores out of TMEM once and hands the S
+// buffer back at once, so the scores of its next tile are computed while it works on this one, and
+// no product waits for another through a shared buffer: S(j+2) follows the read of S(j), PV(j)
+// follows P(j).
 #pragma once
 #include <type_traits>
 
@@ -25,6 +26,10 @@ constexpr int kFwdThreads = 384;
 constexpr int kFwdEwWarp0 = 4;   // first softmax warp
 constexpr int kFwdEwWarps = 8;
 constexpr float kRescaleThreshold = 8.0f;  // lazy O rescale: only when the row max grows by > 2^8
+constexpr int kFwdPolyChains = 0;     // of every four pairs of scores, this many take 2^x from the FMA pipes (ex2_poly_x2)
+constexpr int kFwdExpTurnChunk = 2;   // a group hands the exp2 unit on after this 32-column chunk (of 0..3) of its tile
+constexpr int kFwdRegsIssue = 56;     // registers per thread of warps 0..3 after the re-partitioning
+constexpr int kFwdRegsSoftmax = 224;  // and of the softmax warps (128 * 80 + 256 * 208 <= 384 * 168)
 
 template <int D>
 struct FwdSmem {
@@ -36,15 +41,27 @@ struct FwdSmem {
     static constexpr uint32_t kV = kK + kKStages * kTileBytes;
     static constexpr uint32_t kOut = kV + kVStages * kTileBytes;  // staging tile of O for the tiled store
     static constexpr uint32_t kTotal = kOut + kTileBytes;
-    static constexpr uint32_t kDynamic = kTotal + 1024;  // slack to align the base to 1024 B
+#ifdef SEGATTN_TRACE
+    static constexpr uint32_t kTraceSlots = 3072;  // debug builds: clock stamps are kept in shared memory until the end
+#else
+    static constexpr uint32_t kTraceSlots = 0;
+#endif
+    static constexpr uint32_t kDynamic = kTotal + 1024 + kTraceSlots * 8;  // 1024: slack to align the base to 1024 B
 };
+
+#ifdef SEGATTN_TRACE
+// In this kernel a stamp goes to shared memory (a global store per stamp would sit in front of the
+// kernel's own fences and distort what is measured); the traced CTA copies the stamps out at the end.
+#undef TRACE
+#define TRACE(cond, idx) do { if (trace_on_ && (cond) && (uint32_t)(idx) < SM::kTraceSlots) { long long t_; asm volatile("mov.u64 %0, %clock64;" : "=l"(t_)); asm volatile("st.shared.b64 [%0], %1;" :: "r"(smem_trace + (uint32_t)(idx) * 8u), "l"(t_)); } } while (0)
+#endif
 
 using FwdItem = WorkItem;
 __device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) { return decode_item(prm, idx); }
 // first visible key tile and number of visible key tiles of a work item
 __device__ __forceinline__ void fwd_item_tiles(const FwdParams& prm, const FwdItem& it, int* t_lo, int* n_tiles) {
     long long jl_lo, jl_hi;
-    q_tile_kv_range(prm.geom, it.qt * kTile, it.cls, false, &jl_lo, &jl_hi);
+    q_tile_kv_range<true>(prm.geom, it.qt * kTile, it.cls, false, &jl_lo, &jl_hi);
     *t_lo = (int)(jl_lo / kTile);
     *n_tiles = jl_hi >= jl_lo ? (int)(jl_hi / kTile) - *t_lo + 1 : 0;
 }
@@ -65,8 +82,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     TRACE_INIT();
     constexpr int NQ = SM::kQStages, NK = SM::kKStages, NV = SM::kVStages;
     enum { kBarQFull = 0, kBarQEmpty = kBarQFull + NQ, kBarKFull = kBarQEmpty + NQ, kBarKEmpty = kBarKFull + NK,
-           kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV, kBarSFull = kBarVEmpty + NV, kBarPFull = kBarSFull + 3,
-           kBarPvDone = kBarPFull + 2, kBarSFree = kBarPvDone + 2, kBarOFull = kBarSFree + 3, kNumBars };
+           kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV, kBarSFull = kBarVEmpty + NV, kBarSFree = kBarSFull + 2,
+           kBarPFull = kBarSFree + 2, kBarExp = kBarPFull + 2, kBarPvDone = kBarExp + 8, kBarOFull = kBarPvDone + 2, kNumBars };
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[kNumBars];
     __shared__ uint32_t tmem_slot;
@@ -83,11 +100,17 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     const uint32_t sOut = smem_base + SM::kOut;
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     const MaskGeom& geo = prm.geom;
+#ifdef SEGATTN_TRACE
+    const uint32_t smem_trace = smem_base + SM::kTotal;
+    if (trace_on_)
+        for (uint32_t i = tid; i < SM::kTraceSlots; i += kFwdThreads)
+            asm volatile("st.shared.b64 [%0], %1;" ::"r"(smem_trace + i * 8u), "l"(0ll));
+#endif
 
     if (tid == 0) {
         prefetch_tmap(&prm.to);
         for (int i = 0; i < kNumBars; ++i)
-            mbar_init(bar(i), (i == kBarPFull || i == kBarPFull + 1) ? kFwdEwWarps / 2 : 1);
+            mbar_init(bar(i), (i >= kBarSFree && i < kBarExp) ? kFwdEwWarps / 2 : 1);  // S-free, P-full: one arrival per warp
         fence_mbar_init();
         prefetch_tmap(&prm.tq);
         prefetch_tmap(&prm.tk);
@@ -102,11 +125,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const uint32_t tS0 = tmem, tO = tmem + 384;
-    auto tS = [&](int gj) { return tS0 + (uint32_t)(gj % 3) * 128; };  // S buffer of global key tile gj
+    const uint32_t tS0 = tmem, tP0 = tmem + 256, tO = tmem + 384;  // S and P buffers of group g at tS0 + 128 g, tP0 + 64 g
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
+        setmaxnreg_dec<kFwdRegsIssue>();
         if (lane == 0) {
             ItemWalk q_walk(blockIdx.x, gridDim.x, prm.n_items);  // runs ahead: the next item whose Q is not requested yet
             int qn_ld = 0;        // Q tiles requested so far
@@ -120,7 +143,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     fwd_item_tiles(prm, it, &t_lo, &n);
                     if (n == 0) continue;
                     const int qs = qn_ld % NQ;
-                    if (!(ok = mbar_wait(bar(kBarQEmpty + qs), ((qn_ld / NQ) & 1) ^ 1, 1))) return;
+                    if (!(ok = mbar_wait<true>(bar(kBarQEmpty + qs), ((qn_ld / NQ) & 1) ^ 1, 1))) return;
                     mbar_expect_tx(bar(kBarQFull + qs), SM::kTileBytes);
                     for (int pnl = 0; pnl < SM::kPanels; ++pnl)
                         tma_load_4d(sQ(qs) + pnl * 16384, &prm.tq, bar(kBarQFull + qs), pnl * 64, it.hq, it.qt * kTile, it.b);
@@ -139,7 +162,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 auto load_k = [&](int j) -> bool {
                     const int gj = g + j;
                     const int s = (int)(gj % NK);
-                    if (!mbar_wait(bar(kBarKEmpty + s), (uint32_t)((gj / NK) & 1) ^ 1, 2)) return false;
+                    if (!mbar_wait<true>(bar(kBarKEmpty + s), (uint32_t)((gj / NK) & 1) ^ 1, 2)) return false;
                     mbar_expect_tx(bar(kBarKFull + s), SM::kTileBytes);
                     for (int pnl = 0; pnl < SM::kPanels; ++pnl)
                         tma_load_4d(sK(s) + pnl * 16384, &prm.tk, bar(kBarKFull + s), pnl * 64, it.slot, (t_lo + n - 1 - j) * kTile,
@@ -149,20 +172,19 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 auto load_v = [&](int j) -> bool {
                     const int gj = g + j;
                     const int s = (int)(gj % NV);
-                    if (!mbar_wait(bar(kBarVEmpty + s), (uint32_t)((gj / NV) & 1) ^ 1, 3)) return false;
+                    if (!mbar_wait<true>(bar(kBarVEmpty + s), (uint32_t)((gj / NV) & 1) ^ 1, 3)) return false;
                     mbar_expect_tx(bar(kBarVFull + s), SM::kTileBytes);
                     for (int pnl = 0; pnl < SM::kPanels; ++pnl)
                         tma_load_4d(sV(s) + pnl * 16384, &prm.tv, bar(kBarVFull + s), pnl * 64, it.slot, (t_lo + n - 1 - j) * kTile,
                                     it.b);
                     return true;
                 };
-                // K runs three tiles ahead of V, as the scores do of the PV products
+                // K runs two tiles ahead of V, as the scores do of the PV products
                 ok = ok && load_k(0);
                 if (ok && n > 1) ok = load_k(1);
-                if (ok && n > 2) ok = load_k(2);
                 for (int j = 0; ok && j < n; ++j) {
-                    ok = load_v(j);
-                    if (ok && j + 3 < n) ok = load_k(j + 3);
+                    if (j + 2 < n) ok = load_k(j + 2);
+                    if (ok) ok = load_v(j);
                 }
                 g += n;
                 advance_q();  // the next item's Q: its buffer is free once this item's last scores are issued
@@ -172,15 +194,15 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         // ---------------- MMA issuer for O += P V (whole warp, uniform control flow; one elected lane issues) -------
         // The two kinds of product are issued by two warps on different schedulers, so that neither
         // waits behind the other's barriers and each has half the issue work.
+        setmaxnreg_dec<kFwdRegsIssue>();
         constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
         static_assert(NV == 2 && NK == 2 && NQ == 1, "ring indices below are written out for these depths");
         int g = 0;  // key tiles of earlier work items (a CTA sees far fewer than 2^31)
         bool ok = true;
         ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
-        // The chain P(j) written -> PV(j) issued -> PV(j) finished -> S(j+3) issued -> S(j+3) finished sets
-        // the pace of the kernel, so what the two issuers execute between a barrier and their first product
-        // is kept short: everything that does not depend on the barrier is worked out before the wait, the
-        // waits of one batch share one vote, and optional completion signals are predicated.
+        // What the two issuers execute between a barrier and their first product is kept short: everything
+        // that does not depend on the barrier is worked out before the wait, the waits of one batch share
+        // one vote, and optional completion signals are predicated.
         for (int item; ok && walk.next(&item);) {
             const FwdItem it = fwd_decode(prm, item);
             int t_lo, n;
@@ -190,26 +212,25 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 const int gj = g + j;
                 const int sv = gj & 1;
                 const uint32_t ph = (uint32_t)(gj >> 1) & 1;
-                const uint32_t a_p = tS0 + (uint32_t)(gj % 3) * 128;
-                const uint32_t b_free = bar(kBarSFree + gj % 3);
+                const uint32_t a_p = tP0 + (uint32_t)sv * 64;
                 const uint64_t vd = make_sdesc(sV(sv), 16384, 1024);
                 // V tile landed, P written (the two barriers share ring position and phase)
-                if (!(ok = warp_wait2(bar(kBarVFull + sv), ph, bar(kBarPFull + sv), ph, 6))) break;
+                if (!(ok = warp_wait2<true>(bar(kBarVFull + sv), ph, bar(kBarPFull + sv), ph, 6))) break;
                 tc_fence_after();
-                TRACE(lane == 0, j * 8 + 4);
+                TRACE(lane == 0, j * 16 + 4);
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k)
                     mma_ts(tO, a_p + k * 8, vd + ((k * 2048) >> 4), idesc_pv, (j > 0) || (k > 0));
-                mma_commit(b_free);  // first: P(j) is consumed, the S buffer may take new scores
+                mma_commit(bar(kBarPvDone + sv));  // P(j) is consumed and O holds tile j
                 mma_commit(bar(kBarVEmpty + sv));
-                mma_commit(bar(kBarPvDone + sv));
                 mma_commit_if(j == n - 1, bar(kBarOFull));  // the item's O is complete
-                TRACE(lane == 0, j * 8 + 5);
+                TRACE(lane == 0, j * 16 + 5);
             }
             g += n;
         }
     } else if (warp == 2) {
         // ---------------- MMA issuer for S = Q K^T (whole warp; one elected lane issues) ----------------
+        setmaxnreg_dec<kFwdRegsIssue>();
         constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, 0, 0);
         int qn = 0;  // work items with visible tiles started so far
         int g = 0;   // key tiles of earlier work items
@@ -221,34 +242,35 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             int t_lo, n;
             fwd_item_tiles(prm, it, &t_lo, &n);
             if (n == 0) continue;
-            if (!(ok = warp_wait(bar(kBarQFull), (uint32_t)qn & 1, 4))) break;
+            if (!(ok = warp_wait<true>(bar(kBarQFull), (uint32_t)qn & 1, 4))) break;
             ++qn;
             for (int j = 0; j < n; ++j) {
                 const int gj = g + j;
-                const int s = gj & 1;
-                const int s3 = gj % 3;
-                const uint32_t d_s = tS0 + (uint32_t)s3 * 128;
+                const int s = gj & 1;  // softmax group of the tile = its S buffer = its place in the K ring
+                const uint32_t d_s = tS0 + (uint32_t)s * 128;
                 const uint64_t kd = make_sdesc(sK(s), 16, 1024);
-                // The S buffer of tile gj held P of tile gj - 3: that PV product has finished (the first
-                // three tiles of a launch find fresh buffers: parity 1 of a new barrier reads complete);
-                // and the K tile has landed.
-                const uint32_t free_ph = gj >= 3 ? (uint32_t)((gj - 3) / 3) & 1 : 1u;
-                if (!(ok = warp_wait2(bar(kBarSFree + s3), free_ph, bar(kBarKFull + s), (uint32_t)(gj >> 1) & 1, 12))) break;
+                // The group has read the scores of tile gj - 2 out of this buffer (the first two tiles of a
+                // launch find fresh buffers: parity 1 of a new barrier reads complete); and the K tile has landed.
+                const uint32_t ph = (uint32_t)(gj >> 1) & 1;
+                if (!(ok = warp_wait2<true>(bar(kBarSFree + s), ph ^ 1, bar(kBarKFull + s), ph, 12))) break;
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = ((k / 4) * 16384 + (k % 4) * 32) >> 4;  // descriptor addresses count 16-byte units
                     mma_ss(d_s, qd + off, kd + off, idesc_qk, k > 0);
                 }
-                mma_commit(bar(kBarSFull + s3));  // first: a softmax group waits for it
+                mma_commit(bar(kBarSFull + s));  // first: a softmax group waits for it
                 mma_commit(bar(kBarKEmpty + s));
                 mma_commit_if(j == n - 1, bar(kBarQEmpty));  // the item's last scores release Q
-                TRACE(lane == 0, j * 8 + 6);
+                TRACE(lane == 0, j * 16 + 6);
             }
             g += n;
         }
-    } else if (warp >= kFwdEwWarp0) {
+    } else if (warp < kFwdEwWarp0) {
+        setmaxnreg_dec<kFwdRegsIssue>();  // the idle warp of the issuing warpgroup
+    } else {
         // ---------------- softmax + epilogue ----------------
+        setmaxnreg_inc<kFwdRegsSoftmax>();
         // Two groups of four warps; thread = query row (all 128 key columns of a tile).  Group 0 takes the
         // key tiles of even global index, group 1 the odd ones, so that one group's maximum pass and
         // hand-offs run under the other group's exponentials.  The running maximum travels from tile to
@@ -271,13 +293,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             const int r = r0 + row;
             const long long p = (long long)geo.q_pos0 + r;
             // visible local key rows of this query row: [vlo, vhi]
-            long long vlo_ll = lo_visible(geo, p, it.cls) - geo.kv_pos0;
+            long long vlo_ll = lo_visible<true>(geo, p, it.cls) - geo.kv_pos0;
             long long vhi_ll = p - geo.kv_pos0;
             if (vlo_ll < 0) vlo_ll = 0;
             if (vhi_ll > geo.kv_len - 1) vhi_ll = geo.kv_len - 1;
             const int vlo = (int)vlo_ll, vhi = (int)vhi_ll;
             // a key tile [c0, c0+128) needs no element mask when every row of the tile sees all of it
-            long long full_lo = lo_visible(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.cls) - geo.kv_pos0;
+            long long full_lo = lo_visible<true>(geo, (long long)geo.q_pos0 + r0 + kTile - 1, it.cls) - geo.kv_pos0;
             long long full_hi = (long long)geo.q_pos0 + r0 - geo.kv_pos0;
             if (full_hi > geo.kv_len - 1) full_hi = geo.kv_len - 1;
 
@@ -288,42 +310,54 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             // (outlier keys) stays a convex combination of value rows.
             float m_used = -INFINITY, l_run = 0.f, c_run = 0.f;
             TRACE(tid == 128, 2048 + qn * 4 + 0);
-            // One key tile of the online softmax.  MASKED is a compile-time flag so that the common,
-            // fully visible tile runs straight-line code.
-            auto softmax_tile = [&](auto masked_c, const int j, const int gj, const int c0) {
-                constexpr bool MASKED = decltype(masked_c)::value;
-                const uint32_t tSj = tS(gj);
-                uint32_t va[32], vb[32];
-                // pass 1: row maximum of the raw scores; the load of chunk c+1 is in flight while chunk c is reduced
-                float mx0 = -INFINITY, mx1 = -INFINITY;
-                tmem_ld_x32(tSj + lane_off, va);
+            // One key tile of the online softmax.  One copy of the code serves masked and fully visible tiles
+            // (the mask is applied to the scores in registers, under a branch): the kernel's instruction
+            // footprint, not the branch, is what costs time here.
+            auto softmax_tile = [&](const bool MASKED, const int j, const int gj, const int c0) {
+                const uint32_t tSj = tS0 + (uint32_t)grp * 128 + lane_off;
+                const uint32_t tPj = tP0 + (uint32_t)grp * 64 + lane_off;
+                // the whole row of scores into registers, then the S buffer goes back to the issuer
+                uint32_t sc[4][32];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t(&cur)[32] = (c & 1) ? vb : va;
-                    uint32_t(&nxt)[32] = (c & 1) ? va : vb;
-                    tmem_wait_ld_dep(cur);
-                    tmem_ld_x32(tSj + lane_off + ((c + 1) & 3) * 32, nxt);  // c == 3: chunk 0 again, for pass 2
-                    if (MASKED) {
+                for (int c = 0; c < 4; ++c) tmem_ld_x32(tSj + c * 32, sc[c]);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int col = c0 + c * 32 + i;
-                            cur[i] = (col >= vlo && col <= vhi) ? cur[i] : 0xff800000u;  // -inf
-                        }
-                    }
+                for (int c = 0; c < 4; ++c) tmem_wait_ld_dep(sc[c]);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarSFree + grp));
+                if (MASKED) {
+                    // visible columns of this row inside the tile: [lo_t, hi_t] (tile-local, compared with constants)
+                    const int lo_t = vlo - c0, hi_t = vhi - c0;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        mx0 = fmax3(mx0, __uint_as_float(cur[i]), __uint_as_float(cur[i + 1]));
-                        mx1 = fmax3(mx1, __uint_as_float(cur[i + 2]), __uint_as_float(cur[i + 3]));
-                    }
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            sc[c][i] = (lo_t <= c * 32 + i && hi_t >= c * 32 + i) ? sc[c][i] : 0xff800000u;  // -inf: its p is 0
                 }
-                const float mx = fmaxf(mx0, mx1);
+                // row maximum of the raw scores
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        mx0 = fmax3(mx0, __uint_as_float(sc[c][i]), __uint_as_float(sc[c][i + 1]));
+                        mx1 = fmax3(mx1, __uint_as_float(sc[c][i + 2]), __uint_as_float(sc[c][i + 3]));
+                        mx2 = fmax3(mx2, __uint_as_float(sc[c][i + 4]), __uint_as_float(sc[c][i + 5]));
+                        mx3 = fmax3(mx3, __uint_as_float(sc[c][i + 6]), __uint_as_float(sc[c][i + 7]));
+                    }
+                // the pairs of maximum chain k are the pairs (i / 2) % 4 == k; the last kFwdPolyChains chains are the
+                // pairs whose exponentials come from the polynomial
+                const float mx_unit = kFwdPolyChains >= 2 ? fmaxf(mx0, mx1) : kFwdPolyChains == 1 ? fmax3(mx0, mx1, mx2)
+                                                                                                : fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                const float mx_poly = kFwdPolyChains >= 2 ? fmaxf(mx2, mx3) : kFwdPolyChains == 1 ? mx3 : -INFINITY;
+                const float mx = fmaxf(mx_unit, mx_poly);
                 // running maximum after the previous tile (the other group's), then this tile's
                 float m_prev = -INFINITY;
                 if (j > 0) {
                     fwd_m_sync((int)((gj - 1) & 1));
                     m_prev = s_m[(gj - 1) & 1][row];
                 }
-                TRACE((tid & 127) == 0, j * 8 + 1);
+                TRACE((tid & 127) == 0, j * 16 + 1);
                 const float m_tile = mx * sl2;  // scale > 0, so the maximum commutes with the scaling
                 const bool grow = m_tile > m_prev + kRescaleThreshold || (m_prev == -INFINITY && m_tile > -INFINITY);
                 const float m_new = grow ? m_tile : m_prev;
@@ -332,6 +366,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     __threadfence_block();
                     fwd_m_arrive((int)(gj & 1));
                 }
+                TRACE((tid & 127) == 0, j * 16 + 12);
                 if (m_new > m_used) {  // bring this group's sums to the current scale
                     const float f = ex2(m_used - m_new);  // 0 when nothing was accumulated yet
                     l_run *= f;
@@ -339,10 +374,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     m_used = m_new;
                 }
                 if (j > 0 && __any_sync(0xffffffffu, grow)) {
-                    // PV(j-1), which accumulates into O, was issued after this tile's scores: wait for it
-                    tmem_wait_ld_dep(va);  // the prefetched chunk 0: drain before reusing the load path
+                    // PV(j-1), which accumulates into O, may still be running: wait for it
                     ok = __all_sync(0xffffffffu,
-                                    mbar_wait(bar(kBarPvDone + (int)((gj - 1) & 1)), (uint32_t)(((gj - 1) >> 1) & 1), 10));
+                                    mbar_wait<true>(bar(kBarPvDone + (int)((gj - 1) & 1)), (uint32_t)(((gj - 1) >> 1) & 1), 10));
                     if (!ok) return;
                     tc_fence_after();
                     const float alpha = grow ? ex2(m_prev - m_new) : 1.f;
@@ -356,38 +390,66 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                         tmem_st_x32(tO + lane_off + c * 32, v);
                     }
                 }
-                // pass 2: p = 2^(s*scale*log2e - m); row sum from the unrounded p; P to TMEM as bf16
+                TRACE((tid & 127) == 0, j * 16 + 13);
+                // this group's P buffer is free: PV(j-2) has read it (long since true as a rule)
+                if (gj >= 2) {
+                    ok = __all_sync(0xffffffffu,
+                                    mbar_wait<true>(bar(kBarPvDone + (int)(gj & 1)), (uint32_t)(((gj - 2) >> 1) & 1), 11));
+                    if (!ok) return;
+                }
+                TRACE((tid & 127) == 0, j * 16 + 14);
+                // The two warps of a scheduler (one of each group) take turns at the exponentials: they share
+                // the scheduler's exp2 unit.  This pass starts when the other warp's pass over tile gj - 1 is
+                // nearly through, so that one group's loads, maximum and hand-overs run under the other's
+                // exponentials instead of beside them.
+                if (kFwdExpTurnChunk >= 0 && gj >= 1) {
+                    ok = __all_sync(0xffffffffu, mbar_wait_poll(bar(kBarExp + (int)((gj - 1) & 1) * 4 + quarter),
+                                                                (uint32_t)(((gj - 1) >> 1) & 1), 13));
+                    if (!ok) return;
+                }
+                TRACE((tid & 127) == 0, j * 16 + 7);
+                // p = 2^(s*scale*log2e - m); row sum from the unrounded p; P to TMEM as bf16
                 const float m_eff = (m_new == -INFINITY) ? 0.f : m_new;
                 const uint64_t nm2 = f32x2(-m_eff, -m_eff);
                 {
-                    const float pm = ex2(fmaf(mx, sl2, -m_eff));  // the tile's largest p, exactly as pass 2 forms it
+                    // the tile's largest p, exactly as formed below (by the exp2 unit or by the polynomial)
+                    const float tm = fmaf(mx, sl2, -m_eff);
+                    float pm = ex2(tm);
+                    if (kFwdPolyChains > 0 && mx_poly > mx_unit) {
+                        float q0, q1;
+                        ex2_poly_x2(f32x2(tm, tm), q0, q1);
+                        pm = q0;
+                    }
                     const uint32_t pr = pack_bf16(pm, 0.f);
                     c_run += __uint_as_float(pr << 16) - pm;
                 }
                 uint64_t acc_a = 0ull, acc_b = 0ull;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    uint32_t(&cur)[32] = (c & 1) ? vb : va;
-                    uint32_t(&nxt)[32] = (c & 1) ? va : vb;
-                    tmem_wait_ld_dep(cur);
-                    if (c < 3) tmem_ld_x32(tSj + lane_off + (c + 1) * 32, nxt);
                     uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-                        const uint64_t t = fma_f32x2(f32x2_bits(cur[i], cur[i + 1]), sl2x2, nm2);
-                        float t0, t1;
-                        f32x2_unpack(t, t0, t1);
-                        float p0 = ex2(t0), p1 = ex2(t1);
-                        if (MASKED) {
-                            const int col = c0 + c * 32 + i;
-                            p0 = (col >= vlo && col <= vhi) ? p0 : 0.f;
-                            p1 = (col + 1 >= vlo && col + 1 <= vhi) ? p1 : 0.f;
+                        const uint64_t t = fma_f32x2(f32x2_bits(sc[c][i], sc[c][i + 1]), sl2x2, nm2);
+                        float p0, p1;
+                        if ((i / 2) % 4 >= 4 - kFwdPolyChains) {
+                            ex2_poly_x2(t, p0, p1);
+                        } else {
+                            float t0, t1;
+                            f32x2_unpack(t, t0, t1);
+                            p0 = ex2(t0);
+                            p1 = ex2(t1);
                         }
                         if (i & 2) acc_b = add_f32x2(acc_b, f32x2(p0, p1));
                         else acc_a = add_f32x2(acc_a, f32x2(p0, p1));
                         pk[i / 2] = pack_bf16(p0, p1);
                     }
-                    tmem_st_x16(tSj + lane_off + c * 16, pk);
+                    tmem_st_x16(tPj + c * 16, pk);
+                    TRACE((tid & 127) == 0, j * 16 + 8 + c);
+                    if (c == kFwdExpTurnChunk) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(kBarExp + grp * 4 + quarter));
+                        if (c < 3) reg_fence32(sc[c < 3 ? c + 1 : 3]);  // the rest of the pass stays behind the hand-over
+                    }
                 }
                 {
                     float s0, s1;
@@ -400,25 +462,18 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 if ((gj & 1) != grp) continue;  // the other group's tile
                 const int c0 = (t_lo + n_tiles - 1 - j) * kTile;
                 const bool masked = !(c0 >= full_lo && c0 + kTile - 1 <= full_hi);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarSFull + (int)(gj % 3)), (uint32_t)((gj / 3) & 1), 8));
+                TRACE((tid & 127) == 0, j * 16 + 3);
+                ok = __all_sync(0xffffffffu, mbar_wait<true>(bar(kBarSFull + grp), (uint32_t)((gj >> 1) & 1), 8));
                 if (!ok) break;
                 tc_fence_after();
-                TRACE((tid & 127) == 0, j * 8 + 0);
-                if (masked) softmax_tile(std::true_type{}, j, gj, c0);
-                else softmax_tile(std::false_type{}, j, gj, c0);
+                TRACE((tid & 127) == 0, j * 16 + 0);
+                softmax_tile(masked, j, gj, c0);
                 if (!ok) break;
                 tmem_wait_st();
-                // this group's previous P has been consumed (keeps the P barrier of this parity at most one
-                // completion ahead of the MMA warp; normally long since true)
-                if (gj >= 2) {
-                    ok = __all_sync(0xffffffffu,
-                                    mbar_wait(bar(kBarPvDone + (int)(gj & 1)), (uint32_t)(((gj - 2) >> 1) & 1), 11));
-                    if (!ok) break;
-                }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPFull + (int)(gj & 1)));
-                TRACE((tid & 127) == 0, j * 8 + 2);
+                if (lane == 0) mbar_arrive(bar(kBarPFull + grp));
+                TRACE((tid & 127) == 0, j * 16 + 2);
             }
             if (!ok) break;
             TRACE(tid == 128, 2048 + qn * 4 + 1);
@@ -442,7 +497,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 l_tot = l_g0 + l_g1;
                 lc_tot = l_tot + (c_g0 + c_g1);
                 // one completion per work item: every PV product of the item has finished
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(kBarOFull), (uint32_t)(qn & 1), 9));
+                ok = __all_sync(0xffffffffu, mbar_wait<true>(bar(kBarOFull), (uint32_t)(qn & 1), 9));
                 if (!ok) break;
                 tc_fence_after();
                 TRACE(tid == 128, 2048 + qn * 4 + 2);
@@ -499,6 +554,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     drain_if_failed();
     tc_fence_before();
     __syncthreads();
+#ifdef SEGATTN_TRACE
+    if (trace_on_)
+        for (uint32_t i = tid; i < SM::kTraceSlots; i += kFwdThreads) {
+            long long t_;
+            asm volatile("ld.shared.b64 %0, [%1];" : "=l"(t_) : "r"(smem_trace + i * 8u));
+            g_trace[i] = t_;
+        }
+#endif
     if (warp == 1) {
         __syncwarp();
         tmem_dealloc(tmem, 512);

@@ -76,20 +76,28 @@ __host__ __device__ inline int seg_index(const MaskGeom& g, long long p) {
     return lo;
 }
 // The given-length forms are kept out of line: they run once per work item, and inlining them into
-// the kernels' per-item code costs the constant-length path registers it needs elsewhere.
+// the kernels' per-item code costs the constant-length path registers it needs elsewhere.  INL = true
+// selects inline copies for code that cannot contain calls (a kernel that re-partitions its register
+// file with setmaxnreg).
 #if defined(__CUDACC__)
 #define SEGATTN_NOINLINE __noinline__
 #else
 #define SEGATTN_NOINLINE
 #endif
-__host__ __device__ SEGATTN_NOINLINE inline long long seg_start_given(const MaskGeom& g, long long p) {
+__host__ __device__ inline long long seg_start_given_body(const MaskGeom& g, long long p) {
     return (long long)g.starts[seg_index(g, p)];
 }
-__host__ __device__ SEGATTN_NOINLINE inline long long tail_start_given(const MaskGeom& g, long long p) {
+__host__ __device__ inline long long tail_start_given_body(const MaskGeom& g, long long p) {
     const int i = seg_index(g, p);
     const long long prev0 = i > 0 ? g.starts[i - 1] : 0;
     const long long a = (long long)g.starts[i] - g.T;
     return a < prev0 ? prev0 : a;
+}
+__host__ __device__ SEGATTN_NOINLINE inline long long seg_start_given(const MaskGeom& g, long long p) {
+    return seg_start_given_body(g, p);
+}
+__host__ __device__ SEGATTN_NOINLINE inline long long tail_start_given(const MaskGeom& g, long long p) {
+    return tail_start_given_body(g, p);
 }
 // one past the last reader of key position j (before the detached-prefix rule)
 __host__ __device__ SEGATTN_NOINLINE inline long long hi_diff_given(const MaskGeom& g, long long j, bool own_only) {
@@ -99,11 +107,14 @@ __host__ __device__ SEGATTN_NOINLINE inline long long hi_diff_given(const MaskGe
     return i + 2 < g.n_starts ? g.starts[i + 2] : kPosInf;   // a tail position: the next segment reads it too
 }
 // start of p's segment
+template <bool INL = false>
 __host__ __device__ inline long long seg_start(const MaskGeom& g, long long p) {
-    return g.n_starts ? seg_start_given(g, p) : seg_of(g, p) * (long long)g.S;
+    if (g.n_starts) return INL ? seg_start_given_body(g, p) : seg_start_given(g, p);
+    return seg_of(g, p) * (long long)g.S;
 }
+template <bool INL = false>
 __host__ __device__ inline long long tail_start(const MaskGeom& g, long long p) {
-    if (g.n_starts) return tail_start_given(g, p);
+    if (g.n_starts) return INL ? tail_start_given_body(g, p) : tail_start_given(g, p);
     long long a = seg_of(g, p) * (long long)g.S - g.T;
     return a < 0 ? 0 : a;
 }
@@ -115,9 +126,10 @@ constexpr int kHeadOwn = 2;    // nothing: a long-range head outside the long-ra
 __host__ __device__ inline bool diff_own_only(const MaskGeom& g, int cls) {
     return cls == kHeadOwn || (cls == kHeadPast && g.flagged_tail_sg);
 }
+template <bool INL = false>
 __host__ __device__ inline long long lo_visible(const MaskGeom& g, long long p, int cls) {
     if (cls == kHeadPast) return 0;
-    return cls == kHeadOwn ? seg_start(g, p) : tail_start(g, p);
+    return cls == kHeadOwn ? seg_start<INL>(g, p) : tail_start<INL>(g, p);
 }
 // one past the last query position that differentiably reads key position j of a head of class cls
 __host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, int cls) {
@@ -128,19 +140,21 @@ __host__ __device__ inline long long hi_diff(const MaskGeom& g, long long j, int
     return (j >= seg_end - g.T) ? seg_end + g.S : seg_end;
 }
 // first key position query position p reads differentiably
+template <bool INL = false>
 __host__ __device__ inline long long lo_diff(const MaskGeom& g, long long p, int cls) {
-    const long long lo = diff_own_only(g, cls) ? seg_start(g, p) : tail_start(g, p);
+    const long long lo = diff_own_only(g, cls) ? seg_start<INL>(g, p) : tail_start<INL>(g, p);
     return lo < g.detach_before ? g.detach_before : lo;
 }
 
 // Local key-row range [jl_lo, jl_hi] (inclusive) that the query tile starting at row r0 can see;
 // empty when jl_hi < jl_lo.
+template <bool INL = false>
 __host__ __device__ inline void q_tile_kv_range(const MaskGeom& g, int r0, int cls, bool diff_only,
                                                 long long* jl_lo, long long* jl_hi) {
     int r_last = r0 + kTile - 1;
     if (r_last > g.Lq - 1) r_last = g.Lq - 1;
     long long p0 = (long long)g.q_pos0 + r0, p1 = (long long)g.q_pos0 + r_last;
-    long long lo = diff_only ? lo_diff(g, p0, cls) : lo_visible(g, p0, cls);
+    long long lo = diff_only ? lo_diff<INL>(g, p0, cls) : lo_visible<INL>(g, p0, cls);
     long long a = lo - g.kv_pos0, b = p1 - g.kv_pos0;
     if (a < 0) a = 0;
     if (b > g.kv_len - 1) b = g.kv_len - 1;

@@ -81,8 +81,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // Waits for the phase with the given parity to complete.  Gives up (returns false) when the
 // library's status word is already set by someone else, or after kWaitLimitNs, in which case
 // it records `site` in the status word.  Callers leave their loops on false.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int site,
-                                            unsigned long long limit_ns = kWaitLimitNs) {
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, int site, unsigned long long limit_ns) {
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -95,9 +94,25 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int s
         }
     }
 }
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int site,
+                                            unsigned long long limit_ns = kWaitLimitNs) {
+    return mbar_wait_spin(bar, parity, site, limit_ns);
+}
+// INL: the slow path inline instead of a call.  Code that runs with a re-partitioned register file
+// (setmaxnreg) cannot contain calls: the register allocator refuses them there.
+template <bool INL = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int site) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, site);
+    if constexpr (INL) return mbar_wait_spin(bar, parity, site, kWaitLimitNs);
+    else return mbar_wait_slow(bar, parity, site);
+}
+
+// The same wait by polling (mbarrier.test_wait never suspends the thread): for hand-overs between warps of
+// one scheduler, where the wake-up after a suspending try_wait costs more than the polling does.
+__device__ __forceinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, int site) {
+    for (uint32_t it = 0; it < 4096u; ++it)
+        if (mbar_test_wait(bar, parity)) return true;
+    return mbar_wait_spin(bar, parity, site, kWaitLimitNs);
 }
 
 // After a failed wait: give this CTA's outstanding bulk copies time to land (bounded) before its
@@ -206,6 +221,12 @@ __device__ __forceinline__ void tmem_wait_ld_dep(uint32_t (&r)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31]) :: "memory");
 }
 
+// Compiler-only fence on 32 registers: what is computed from them afterwards cannot be scheduled
+// before this point (no instruction is emitted).
+__device__ __forceinline__ void reg_fence32(uint32_t (&r)[32]) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31]) :: "memory");
+}
+
 // ---- tcgen05: MMA ----------------------------------------------------------------------------
 // Instruction descriptor of kind::f16 with bf16 A/B and f32 accumulation:
 // [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format (1 = bf16),
@@ -263,21 +284,34 @@ __device__ __forceinline__ void mma_commit_if(bool pred, uint32_t bar) {
         : "memory");
 }
 // A bounded wait executed by a whole warp, with a warp-uniform result.
+template <bool INL = false>
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, int site) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, site));
+    return __all_sync(0xffffffffu, mbar_wait<INL>(bar, parity, site));
 }
 // Bounded waits of a whole warp on two or three barriers at once: one poll of each, one vote and
 // one branch when all of them have completed already, which is the common case for an MMA issuer.
+template <bool INL = false>
 __device__ __forceinline__ bool warp_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b, int site) {
     const bool done = mbar_try_wait(bar_a, par_a) & mbar_try_wait(bar_b, par_b);
     if (__all_sync(0xffffffffu, done)) return true;
-    return warp_wait(bar_a, par_a, site) && warp_wait(bar_b, par_b, site);
+    return warp_wait<INL>(bar_a, par_a, site) && warp_wait<INL>(bar_b, par_b, site);
 }
 __device__ __forceinline__ bool warp_wait3(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b, uint32_t bar_c,
                                            uint32_t par_c, int site) {
     const bool done = mbar_try_wait(bar_a, par_a) & mbar_try_wait(bar_b, par_b) & mbar_try_wait(bar_c, par_c);
     if (__all_sync(0xffffffffu, done)) return true;
     return warp_wait(bar_a, par_a, site) && warp_wait(bar_b, par_b, site) && warp_wait(bar_c, par_c, site);
+}
+
+// Re-partitioning of the register file between the warpgroups of a CTA (all four warps of a warpgroup
+// execute the same instruction): the issuing warps hand registers to the element-wise warps.
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 // ---- small numeric helpers ---------------------------------------------------------------------
