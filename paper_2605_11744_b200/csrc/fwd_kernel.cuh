@@ -28,6 +28,8 @@ constexpr int kFwdEwWarps = 8;
 constexpr float kRescaleThreshold = 8.0f;  // lazy O rescale: only when the row max grows by > 2^8
 constexpr int kFwdPolyChains = 0;     // of every four pairs of scores, this many take 2^x from the FMA pipes (ex2_poly_x2)
 constexpr int kFwdExpTurnChunk = 2;   // a group hands the exp2 unit on after this 32-column chunk (of 0..3) of its tile
+constexpr int kFwdRing = 8;           // decoded work items in flight between the scheduling warp and the other roles
+constexpr int kFwdDescReaders = 12;   // readers of a decoded item: producer (twice: Q cursor and K/V cursor), two issuers, eight softmax warps
 constexpr int kFwdRegsIssue = 56;     // registers per thread of warps 0..3 after the re-partitioning
 constexpr int kFwdRegsSoftmax = 224;  // and of the softmax warps (128 * 80 + 256 * 208 <= 384 * 168)
 
@@ -56,6 +58,12 @@ struct FwdSmem {
 #define TRACE(cond, idx) do { if (trace_on_ && (cond) && (uint32_t)(idx) < SM::kTraceSlots) { long long t_; asm volatile("mov.u64 %0, %clock64;" : "=l"(t_)); asm volatile("st.shared.b64 [%0], %1;" :: "r"(smem_trace + (uint32_t)(idx) * 8u), "l"(t_)); } } while (0)
 #endif
 
+// A decoded work item as the scheduling warp publishes it in shared memory (32 bytes): the item and
+// its visible key tiles [t_lo, t_lo + n).  n = 0: nothing visible (the rows are written as zeros);
+// n < 0: end of this CTA's list.
+struct FwdDesc {
+    int b, hq, slot, qt, cls, t_lo, n;
+};
 using FwdItem = WorkItem;
 __device__ __forceinline__ FwdItem fwd_decode(const FwdParams& prm, int idx) { return decode_item(prm, idx); }
 // first visible key tile and number of visible key tiles of a work item
@@ -74,6 +82,13 @@ __device__ __forceinline__ void fwd_m_sync(int parity) { asm volatile("bar.sync 
 // barrier of all eight softmax warps
 __device__ __forceinline__ void fwd_groups_sync() { asm volatile("bar.sync 4, 256;" ::: "memory"); }
 
+// score := -inf (its p is then 0) unless lo <= col <= hi; col is a constant: two compares and a select
+__device__ __forceinline__ void mask_score(uint32_t& x, int lo, int hi, int col) {
+    asm("{\n\t.reg .pred p;\n\tsetp.gt.s32 p, %1, %3;\n\tsetp.lt.or.s32 p, %2, %3, p;\n\tselp.b32 %0, 0xff800000, %0, p;\n\t}"
+        : "+r"(x)
+        : "r"(lo), "r"(hi), "r"(col));
+}
+
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __grid_constant__ FwdParams prm) {
     using SM = FwdSmem<D>;
@@ -83,12 +98,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     constexpr int NQ = SM::kQStages, NK = SM::kKStages, NV = SM::kVStages;
     enum { kBarQFull = 0, kBarQEmpty = kBarQFull + NQ, kBarKFull = kBarQEmpty + NQ, kBarKEmpty = kBarKFull + NK,
            kBarVFull = kBarKEmpty + NK, kBarVEmpty = kBarVFull + NV, kBarSFull = kBarVEmpty + NV, kBarSFree = kBarSFull + 2,
-           kBarPFull = kBarSFree + 2, kBarExp = kBarPFull + 2, kBarPvDone = kBarExp + 8, kBarOFull = kBarPvDone + 2, kNumBars };
+           kBarPFull = kBarSFree + 2, kBarExp = kBarPFull + 2, kBarPvDone = kBarExp + 8, kBarOFull = kBarPvDone + 2, kBarDescFull = kBarOFull + 1,
+           kBarDescEmpty = kBarDescFull + kFwdRing, kNumBars = kBarDescEmpty + kFwdRing };
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[kNumBars];
     __shared__ uint32_t tmem_slot;
     __shared__ float s_m[2][kTile];       // [tile parity][row]: running row maximum after that tile
     __shared__ float s_fin[2][3][kTile];  // [group][m, l, c][row]: the groups' partial sums, once per work item
+    __shared__ __align__(16) int s_desc[kFwdRing][8];  // ring of decoded work items (FwdDesc)
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -110,7 +127,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     if (tid == 0) {
         prefetch_tmap(&prm.to);
         for (int i = 0; i < kNumBars; ++i)
-            mbar_init(bar(i), (i >= kBarSFree && i < kBarExp) ? kFwdEwWarps / 2 : 1);  // S-free, P-full: one arrival per warp
+            mbar_init(bar(i), (i >= kBarSFree && i < kBarExp) ? kFwdEwWarps / 2  // S-free, P-full: one arrival per warp
+                              : i >= kBarDescEmpty                ? kFwdDescReaders
+                                                                  : 1);
         fence_mbar_init();
         prefetch_tmap(&prm.tq);
         prefetch_tmap(&prm.tk);
@@ -126,22 +145,38 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     const uint32_t tS0 = tmem, tP0 = tmem + 256, tO = tmem + 384;  // S and P buffers of group g at tS0 + 128 g, tP0 + 64 g
+    // The k-th work item of this CTA as the scheduling warp decoded it (called by a whole warp or by one
+    // lane of it; `leader` marks the one thread that hands the ring slot back).  False: a wait gave up.
+    auto read_desc = [&](int k, FwdDesc* d, bool whole_warp, bool leader) -> bool {
+        const int rs = k % kFwdRing;
+        if (!mbar_wait<true>(bar(kBarDescFull + rs), (uint32_t)(k / kFwdRing) & 1, 14)) return false;
+        const uint32_t a = smem_u32(&s_desc[rs][0]);
+        int pad;
+        ld_shared_v4(a, d->b, d->hq, d->slot, d->qt);
+        ld_shared_v4(a + 16, d->cls, d->t_lo, d->n, pad);
+        if (whole_warp) __syncwarp();
+        if (leader) mbar_arrive(bar(kBarDescEmpty + rs));
+        return true;
+    };
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         setmaxnreg_dec<kFwdRegsIssue>();
         if (lane == 0) {
-            ItemWalk q_walk(blockIdx.x, gridDim.x, prm.n_items);  // runs ahead: the next item whose Q is not requested yet
+            int kq = 0;           // Q cursor: runs ahead, the next item whose Q is not requested yet
+            bool q_more = true;   // the Q cursor has not reached the end of the list
             int qn_ld = 0;        // Q tiles requested so far
             bool ok = true;
             // request the Q tile of the next work item that has visible key tiles, if there is one
             auto advance_q = [&]() {
-                int qi;
-                while (ok && q_walk.next(&qi)) {
-                    const FwdItem it = fwd_decode(prm, qi);
-                    int t_lo, n;
-                    fwd_item_tiles(prm, it, &t_lo, &n);
-                    if (n == 0) continue;
+                while (ok && q_more) {
+                    FwdDesc it;
+                    if (!(ok = read_desc(kq++, &it, false, true))) return;
+                    if (it.n < 0) {
+                        q_more = false;
+                        return;
+                    }
+                    if (it.n == 0) continue;
                     const int qs = qn_ld % NQ;
                     if (!(ok = mbar_wait<true>(bar(kBarQEmpty + qs), ((qn_ld / NQ) & 1) ^ 1, 1))) return;
                     mbar_expect_tx(bar(kBarQFull + qs), SM::kTileBytes);
@@ -153,11 +188,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             };
             int g = 0;  // key tiles requested so far (all work items; far fewer than 2^31)
             advance_q();
-            ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
-        for (int item; ok && walk.next(&item);) {
-                const FwdItem it = fwd_decode(prm, item);
-                int t_lo, n;
-                fwd_item_tiles(prm, it, &t_lo, &n);
+            for (int kd = 0; ok; ++kd) {
+                FwdDesc it;
+                if (!(ok = read_desc(kd, &it, false, true)) || it.n < 0) break;
+                const int t_lo = it.t_lo, n = it.n;
                 if (n == 0) continue;
                 auto load_k = [&](int j) -> bool {
                     const int gj = g + j;
@@ -199,14 +233,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         static_assert(NV == 2 && NK == 2 && NQ == 1, "ring indices below are written out for these depths");
         int g = 0;  // key tiles of earlier work items (a CTA sees far fewer than 2^31)
         bool ok = true;
-        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
         // What the two issuers execute between a barrier and their first product is kept short: everything
         // that does not depend on the barrier is worked out before the wait, the waits of one batch share
         // one vote, and optional completion signals are predicated.
-        for (int item; ok && walk.next(&item);) {
-            const FwdItem it = fwd_decode(prm, item);
-            int t_lo, n;
-            fwd_item_tiles(prm, it, &t_lo, &n);
+        for (int kd = 0; ok; ++kd) {
+            FwdDesc it;
+            ok = __all_sync(0xffffffffu, read_desc(kd, &it, true, lane == 0));
+            if (!ok || it.n < 0) break;
+            const int n = it.n;
             if (n == 0) continue;
             for (int j = 0; j < n; ++j) {
                 const int gj = g + j;
@@ -236,11 +270,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         int g = 0;   // key tiles of earlier work items
         bool ok = true;
         const uint64_t qd = make_sdesc(sQ(0), 16, 1024);
-        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
-        for (int item; ok && walk.next(&item);) {
-            const FwdItem it = fwd_decode(prm, item);
-            int t_lo, n;
-            fwd_item_tiles(prm, it, &t_lo, &n);
+        for (int kd = 0; ok; ++kd) {
+            FwdDesc it;
+            ok = __all_sync(0xffffffffu, read_desc(kd, &it, true, lane == 0));
+            if (!ok || it.n < 0) break;
+            const int n = it.n;
             if (n == 0) continue;
             if (!(ok = warp_wait<true>(bar(kBarQFull), (uint32_t)qn & 1, 4))) break;
             ++qn;
@@ -267,7 +301,27 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
             g += n;
         }
     } else if (warp < kFwdEwWarp0) {
-        setmaxnreg_dec<kFwdRegsIssue>();  // the idle warp of the issuing warpgroup
+        // ---------------- scheduling warp: decodes this CTA's work items once, for every other role ----------------
+        setmaxnreg_dec<kFwdRegsIssue>();
+        if (lane == 0) {
+            ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
+            bool more = true;
+            for (int k = 0; more; ++k) {
+                const int rs = k % kFwdRing;
+                // every reader has taken the item that was in this slot (a fresh barrier reads complete for parity 1)
+                if (!mbar_wait<true>(bar(kBarDescEmpty + rs), ((uint32_t)(k / kFwdRing) & 1) ^ 1, 15)) break;
+                int item, t_lo = 0, n = -1;
+                FwdItem it = {0, 0, 0, 0, 0};
+                if ((more = walk.next(&item))) {
+                    it = fwd_decode(prm, item);
+                    fwd_item_tiles(prm, it, &t_lo, &n);
+                }
+                const uint32_t a = smem_u32(&s_desc[rs][0]);
+                st_shared_v4(a, (uint32_t)it.b, (uint32_t)it.hq, (uint32_t)it.slot, (uint32_t)it.qt);
+                st_shared_v4(a + 16, (uint32_t)it.cls, (uint32_t)t_lo, (uint32_t)n, 0u);
+                mbar_arrive(bar(kBarDescFull + rs));  // release: the stores above are visible to whoever sees the arrival
+            }
+        }
     } else {
         // ---------------- softmax + epilogue ----------------
         setmaxnreg_inc<kFwdRegsSoftmax>();
@@ -284,11 +338,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
         int g = 0;   // key tiles of earlier work items (a CTA sees far fewer than 2^31)
         int qn = 0;  // earlier work items that had visible tiles
         bool ok = true;
-        ItemWalk walk(blockIdx.x, gridDim.x, prm.n_items);
-        for (int item; ok && walk.next(&item);) {
-            const FwdItem it = fwd_decode(prm, item);
-            int t_lo, n_tiles;
-            fwd_item_tiles(prm, it, &t_lo, &n_tiles);
+        for (int kd = 0; ok; ++kd) {
+            FwdDesc it;
+            ok = __all_sync(0xffffffffu, read_desc(kd, &it, true, lane == 0));
+            if (!ok || it.n < 0) break;
+            const int t_lo = it.t_lo, n_tiles = it.n;
             const int r0 = it.qt * kTile;
             const int r = r0 + row;
             const long long p = (long long)geo.q_pos0 + r;
@@ -331,8 +385,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            sc[c][i] = (lo_t <= c * 32 + i && hi_t >= c * 32 + i) ? sc[c][i] : 0xff800000u;  // -inf: its p is 0
+                        for (int i = 0; i < 32; ++i) mask_score(sc[c][i], lo_t, hi_t, c * 32 + i);
                 }
                 // row maximum of the raw scores
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -380,7 +433,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                     if (!ok) return;
                     tc_fence_after();
                     const float alpha = grow ? ex2(m_prev - m_new) : 1.f;
-#pragma unroll
+#pragma unroll 1  // rare (the row maximum has grown by more than the threshold): kept small, not fast
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t v[32];
                         tmem_ld_x32(tO + lane_off + c * 32, v);
@@ -403,8 +456,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __gr
                 // nearly through, so that one group's loads, maximum and hand-overs run under the other's
                 // exponentials instead of beside them.
                 if (kFwdExpTurnChunk >= 0 && gj >= 1) {
-                    ok = __all_sync(0xffffffffu, mbar_wait_poll(bar(kBarExp + (int)((gj - 1) & 1) * 4 + quarter),
-                                                                (uint32_t)(((gj - 1) >> 1) & 1), 13));
+                    ok = __all_sync(0xffffffffu, mbar_wait<true>(bar(kBarExp + (int)((gj - 1) & 1) * 4 + quarter),
+                                                                 (uint32_t)(((gj - 1) >> 1) & 1), 13));
                     if (!ok) return;
                 }
                 TRACE((tid & 127) == 0, j * 16 + 7);

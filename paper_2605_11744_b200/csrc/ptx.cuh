@@ -99,20 +99,23 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int s
     return mbar_wait_spin(bar, parity, site, limit_ns);
 }
 // INL: the slow path inline instead of a call.  Code that runs with a re-partitioned register file
-// (setmaxnreg) cannot contain calls: the register allocator refuses them there.
+// (setmaxnreg) cannot contain calls: the register allocator refuses them there.  The inline form is kept
+// to a few instructions (a kernel's instruction footprint costs time): it bounds the wait by a count of
+// polls instead of the timer.  One mbarrier.try_wait that does not succeed suspends the thread for about
+// 1.5 us on this part, so 2^20 polls are about 1.5 s.
+constexpr uint32_t kWaitLimitPolls = 1u << 20;
 template <bool INL = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int site) {
     if (mbar_try_wait(bar, parity)) return true;
-    if constexpr (INL) return mbar_wait_spin(bar, parity, site, kWaitLimitNs);
-    else return mbar_wait_slow(bar, parity, site);
-}
-
-// The same wait by polling (mbarrier.test_wait never suspends the thread): for hand-overs between warps of
-// one scheduler, where the wake-up after a suspending try_wait costs more than the polling does.
-__device__ __forceinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, int site) {
-    for (uint32_t it = 0; it < 4096u; ++it)
-        if (mbar_test_wait(bar, parity)) return true;
-    return mbar_wait_spin(bar, parity, site, kWaitLimitNs);
+    if constexpr (INL) {
+#pragma unroll 1
+        for (uint32_t it = 0; it < kWaitLimitPolls; ++it)
+            if (mbar_try_wait(bar, parity)) return true;
+        atomicCAS(&g_device_status, 0, (4 << 8) | (site & 0xff));
+        return false;
+    } else {
+        return mbar_wait_slow(bar, parity, site);
+    }
 }
 
 // After a failed wait: give this CTA's outstanding bulk copies time to land (bounded) before its
@@ -154,6 +157,9 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // one 16-byte store to shared memory
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void ld_shared_v4(uint32_t addr, int& x, int& y, int& z, int& w) {
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
