@@ -84,7 +84,7 @@ def group_slices(mask, g):
 def oracle_window(x, w, b, c, hq, seg_lo, n_seg=2):
     """Oracle forward + backward for batch b, KV head c (query heads hq) on the queries of
     segments [seg_lo, seg_lo + n_seg) against every key before the window's end.  `keys` is the range whose
-    dK/dV are complete: the window's keys without its last segment (whose tail the next segment also reads),
+    dK/dV are complete: the window's keys without the last T of them (the tail the next segment also reads),
     or all of them when the window ends the sequence."""
     S = w.S
     r0, r1 = seg_lo * S, min(w.L, (seg_lo + n_seg) * S)
@@ -97,7 +97,7 @@ def oracle_window(x, w, b, c, hq, seg_lo, n_seg=2):
     if "dO" in x:
         dO = f64(x["dO"][b:b + 1, r0:r1, hq])
         dQ, dK, dV = oracle.bwd(Q, K, V, dO, S, w.T, m, scale=w.sm_scale, q_pos0=r0)
-        k1 = r1 if r1 == w.L else max(r0 + S, r1 - S)
+        k1 = r1 if r1 == w.L else r1 - w.T
         out.update(dQ=dQ, dK=dK[:, r0:k1], dV=dV[:, r0:k1], keys=slice(r0, k1))
     return out
 
