@@ -37,13 +37,13 @@ UNIT = "TFLOP/s"
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel on the
 # benchmark workload, taken from the ncu captures summarised under profiles/; None = not captured.
 NCU_TRAFFIC_BYTES = {
-    ("cfg2_gqa16k", "fwd"): 643414144,
+    ("cfg2_gqa16k", "fwd"): 641431168,
     ("cfg2_gqa16k", "dq"): 929728256,
     ("cfg2_gqa16k", "dkv"): 800741376,
-    ("cfg3_outlier32k", "fwd"): 846842240,
+    ("cfg3_outlier32k", "fwd"): 828632192,
     ("cfg3_outlier32k", "dq"): 1199171072,
     ("cfg3_outlier32k", "dkv"): 801214208,
-    ("cfg5_S1024_T256_f0", "fwd"): 2441578624,
+    ("cfg5_S1024_T256_f0", "fwd"): 2398129920,
     ("cfg5_S1024_T256_f0", "dq"): 3496404608,
     ("cfg5_S1024_T256_f0", "dkv"): 2771600896,
 }
