@@ -82,13 +82,6 @@ __device__ __forceinline__ void fwd_m_sync(int parity) { asm volatile("bar.sync 
 // barrier of all eight softmax warps
 __device__ __forceinline__ void fwd_groups_sync() { asm volatile("bar.sync 4, 256;" ::: "memory"); }
 
-// score := -inf (its p is then 0) unless lo <= col <= hi; col is a constant: two compares and a select
-__device__ __forceinline__ void mask_score(uint32_t& x, int lo, int hi, int col) {
-    asm("{\n\t.reg .pred p;\n\tsetp.gt.s32 p, %1, %3;\n\tsetp.lt.or.s32 p, %2, %3, p;\n\tselp.b32 %0, 0xff800000, %0, p;\n\t}"
-        : "+r"(x)
-        : "r"(lo), "r"(hi), "r"(col));
-}
-
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1) seg_attn_fwd_kernel(const __grid_constant__ FwdParams prm) {
     using SM = FwdSmem<D>;

@@ -396,4 +396,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
+// score := -inf (its p is then 0) unless lo <= col <= hi; col is a constant: two compares and a select
+__device__ __forceinline__ void mask_score(uint32_t& x, int lo, int hi, int col) {
+    asm("{\n\t.reg .pred p;\n\tsetp.gt.s32 p, %1, %3;\n\tsetp.lt.or.s32 p, %2, %3, p;\n\tselp.b32 %0, 0xff800000, %0, p;\n\t}"
+        : "+r"(x)
+        : "r"(lo), "r"(hi), "r"(col));
+}
+
 }  // namespace segattn
