@@ -190,20 +190,20 @@ segattn_status seg_prefill_step(seg_prefill_handle* h, const void* Qseg, const v
  * in particular a shorter last segment.  The segment tensors hold Lseg rows per batch element and are addressed with
  * the strides given at creation; LSE_seg is [B][Hq][Lseg].  The carried tail of a segment shorter than T is the whole
  * segment (never more than one segment back), as with seg_attn_params.seg_starts, whose whole-sequence forward this
- * reproduces row for row.  seg_prefill_step(h, ...) is seg_prefill_step_len(h, S, ...).  seg_prefill_step_bwd takes
- * constant-length streams only: after a step with Lseg != S, or after any step that followed one, it returns
- * SEGATTN_ERR_INVALID. */
+ * reproduces row for row.  seg_prefill_step(h, ...) is seg_prefill_step_len(h, S, ...). */
 segattn_status seg_prefill_step_len(seg_prefill_handle* h, int32_t Lseg, const void* Qseg, const void* Kseg,
                                     const void* Vseg, void* Oseg, float* LSEseg, void* stream);
 /* Backward of the segment stepped last (the streamed form of training with truncation depth 1: a
  * segment is run forward, its loss is differentiated, and credit stops where the carried state
  * entered - definition of the K-truncated objective with K = 1).  Valid after seg_prefill_step and
  * before the next one; the state still holds what that step attended over.  Qseg, Oseg, dOseg and
- * dQseg are [B][S][Hq][d] with the strides given at creation, LSEseg as returned by the step.
+ * dQseg hold the Lseg rows of that step per batch element ([B][S][Hq][d] for a full segment) with the strides
+ * given at creation, LSEseg as returned by the step.
  * dKctx and dVctx are contiguous bf16 [B][T+S][Hkv][d]: the gradients of the key/value rows at
- * global positions [i*S - T, i*S + S) - the previous segment's carried tail, then the segment itself
- * (rows before position 0 are zero).  Older rows of past-access heads are read forward-only and get
- * none.  The caller adds the first T rows to the previous segment's gradients.  `workspace`: DEVICE,
+ * global positions [pos - T, pos + Lseg), pos the segment's start - the T positions in front of the segment, of
+ * which the previous segment's carried tail (its last min(T, length) positions) can be non-zero, then the segment
+ * itself; rows before position 0 and the S - Lseg rows after a shorter segment are zero.  Older rows of past-access
+ * heads are read forward-only and get none.  The caller adds the first T rows to the previous segment's gradients.  `workspace`: DEVICE,
  * 256-byte aligned, at least seg_prefill_bwd_workspace_bytes(h) bytes.  SEGATTN_ERR_INVALID when no segment
  * has been stepped yet or a pointer is null or misaligned, SEGATTN_ERR_WORKSPACE for the workspace; the state
  * is not modified. */

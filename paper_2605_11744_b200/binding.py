@@ -395,14 +395,16 @@ class Prefill:
         return out, LSE
 
     def step_bwd(self, Qseg, Oseg, LSEseg, dOseg, stream=None):
-        """Backward of the segment stepped last: dQ [B,S,Hq,d] and dK, dV [B,T+S,Hkv,d] for the key/value rows
-        [previous tail ; segment] - the C entry point `seg_prefill_step_bwd`."""
+        """Backward of the segment stepped last: dQ [B,Lseg,Hq,d] and dK, dV [B,T+S,Hkv,d] for the key/value rows
+        [T positions in front of the segment ; segment ; zeros] - the C entry point `seg_prefill_step_bwd`."""
         _need_cuda_bf16(Qseg, Oseg, dOseg)
         p = self.params
+        Lseg = Qseg.shape[1]
         for t in (Qseg, Oseg, dOseg):
-            if tuple(t.shape) != (p.B, p.S, p.Hq, p.d) or not t.is_contiguous():
-                raise ValueError("segment tensors must be contiguous [B,S,Hq,d]")
-        dQ = torch.empty_like(Qseg)
+            if not (t.dim() == 4 and tuple(t.shape) == (p.B, Lseg, p.Hq, p.d) and t.stride(3) == 1 and t.stride(2) == p.d and
+                    t.stride(1) == p.Hq * p.d and (p.B == 1 or t.stride(0) == p.S * p.Hq * p.d)):
+                raise ValueError("segment tensors must be [B, Lseg, Hq, d] with the strides of a contiguous [B, S, Hq, d]")
+        dQ = torch.empty((p.B, p.S, p.Hq, p.d), dtype=torch.bfloat16, device=Qseg.device)[:, :Lseg]
         dK = torch.empty((p.B, p.T + p.S, p.Hkv, p.d), dtype=torch.bfloat16, device=Qseg.device)
         dV = torch.empty_like(dK)
         need = int(lib().seg_prefill_bwd_workspace_bytes(self._h))

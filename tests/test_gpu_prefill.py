@@ -236,13 +236,62 @@ def test_streamed_segments_of_unequal_lengths(B, Hq, Hkv, d, S, T, mask, lengths
         assert (O1.float() - O2.float()).abs().max() <= 2e-2
 
 
-def test_streamed_backward_refuses_unequal_lengths_and_oversized_segments():
+@pytest.mark.parametrize("B,Hq,Hkv,d,S,T,mask,lengths", [
+    (1, 4, 2, 128, 256, 128, [0, 1], [256, 256, 100]),                 # a shorter last segment
+    (2, 4, 2, 128, 256, 128, [0, 1], [256, 128, 256, 128]),            # unequal lengths on tile boundaries, two batch elements
+    (1, 2, 2, 128, 300, 100, [0, 1], [300, 37, 1, 250, 64]),           # nothing aligned; segments shorter than the tail
+    (1, 6, 3, 64, 200, 200, [2, 1, 0], [64, 200, 150, 3]),             # d = 64, all head classes, T = S
+])
+def test_streamed_backward_over_segments_of_unequal_lengths(B, Hq, Hkv, d, S, T, mask, lengths):
+    # The backward of each streamed step, for segments of lengths m_i: every term against the oracle (loss of that
+    # segment alone over the same segment starts), and the terms added up against the whole-sequence backward.
+    from util import assert_grads_close
+    L = sum(lengths)
+    starts = [0] + [int(v) for v in np.cumsum(lengths)[:-1]]
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=L + S + 7)
+    Qf, Kf, Vf, dOf = f64(Q), f64(K), f64(V), f64(dO)
+    pf = sa.Prefill(B, S, T, Hq, Hkv, d, L, mask)
+    dQ = torch.empty_like(Q)
+    dK = torch.zeros(B, L, Hkv, d, dtype=torch.float32, device="cuda")
+    dV = torch.zeros_like(dK)
+    bufs = [torch.empty(B, S, t.shape[2], d, dtype=torch.bfloat16, device="cuda") for t in (Q, K, V, dO)]
+    s0 = 0
+    for i, m in enumerate(lengths):
+        views = []
+        for buf, t in zip(bufs, (Q, K, V, dO)):
+            buf[:, :m] = t[:, s0:s0 + m]
+            views.append(buf[:, :m])
+        q, k, v, do = views
+        o, lse = pf.step(q, k, v)
+        gq, gk, gv = pf.step_bwd(q, o, lse, do)
+        sa.poll_status()
+        assert gq.shape == (B, m, Hq, d) and gk.shape == (B, T + S, Hkv, d)
+        dQ[:, s0:s0 + m] = gq
+        lo = s0 - T                      # global position of row 0 of gk / gv
+        cut = max(0, -lo)
+        assert not gk[:, :cut].any() and not gv[:, :cut].any()            # rows before position 0
+        assert not gk[:, T + m:].any() and not gv[:, T + m:].any()        # rows after a shorter segment
+        dK[:, lo + cut:s0 + m] += gk[:, cut:T + m].float()
+        dV[:, lo + cut:s0 + m] += gv[:, cut:T + m].float()
+        # this segment's term against the oracle: the loss of segment i alone, sequence up to its end
+        hi = s0 + m
+        dOw = np.zeros_like(dOf[:, :hi])
+        dOw[:, s0:hi] = dOf[:, s0:hi]
+        rq, rk, rv = oracle.bwd(Qf[:, :hi], Kf[:, :hi], Vf[:, :hi], dOw, 1, T, mask, seg_starts=starts[:i + 1])
+        assert not rk[:, :lo + cut].any()          # nothing in front of the T rows before the segment receives gradient
+        assert_grads_close((gq, gk[:, cut:T + m], gv[:, cut:T + m]), (rq[:, s0:hi], rk[:, lo + cut:], rv[:, lo + cut:]),
+                           "segment %d" % i)
+        s0 += m
+    pf.close()
+    ref = oracle.bwd(Qf, Kf, Vf, dOf, 1, T, mask, seg_starts=starts)
+    assert_grads_close((dQ, dK, dV), ref, "sum over segments of unequal lengths")
+
+
+def test_streamed_driver_refuses_oversized_segments():
     B, Hq, Hkv, d, S, T = 1, 2, 1, 128, 128, 64
     Q, K, V, dO = rand_inputs(B, 256, Hq, Hkv, d, seed=4)
     pf = sa.Prefill(B, S, T, Hq, Hkv, d, 256, [0])
     o, l = pf.step(Q[:, :100], K[:, :100], V[:, :100])
-    with pytest.raises(sa.SegAttnError):
-        pf.step_bwd(Q[:, :128].contiguous(), Q[:, :128].contiguous(), torch.zeros(B, Hq, S, device="cuda"), dO[:, :128].contiguous())
     with pytest.raises(ValueError):
         pf.step(Q[:, :200], K[:, :200], V[:, :200])     # longer than S
     h = pf._h
