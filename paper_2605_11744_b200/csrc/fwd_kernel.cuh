@@ -4,10 +4,11 @@
 // Persistent: one CTA per SM walks a static list of work items (one 128-row query tile of one
 // (batch, query head) each), heaviest items first, dealt round-robin to the CTAs.
 // Roles (384 threads): warp 0 = TMA producer, warp 1 = tcgen05 issuer of the PV products and TMEM
-// owner, warp 2 = tcgen05 issuer of the score products,
+// owner, warp 2 = tcgen05 issuer of the score products, warp 3 = scheduling warp (decodes the CTA's
+// work items once and hands them to every other role through a ring in shared memory),
 // warps 4..7 and 8..11 = two softmax groups (thread = query row) that take the key tiles of even
 // and odd index in turn and pass the running row maximum on through shared memory, then share the
-// epilogue; warp 3 idle.  The issuing warpgroup gives most of its registers to the softmax groups,
+// epilogue.  The issuing warpgroup gives most of its registers to the softmax groups,
 // whose threads hold a whole row of scores (128 values) in registers.
 // TMEM (512 columns): one S buffer per softmax group at [0,256), one P buffer (bf16) per group at
 // [256,384), O at [384,384+D).  A group reads its tile's scores out of TMEM once and hands the S
