@@ -240,6 +240,24 @@ def test_empty_and_degenerate_shapes():
     assert torch.count_nonzero(dQ[:, 128:]) == 0
 
 
+def test_more_work_items_per_block_than_the_item_ring_holds_with_keyless_items_among_them():
+    # 1536 work items (about ten per persistent block, more than the ring of decoded items between the scheduling
+    # warp and the other roles holds), of which the later query tiles of the local head have no key in reach
+    # (the keys end half way): those items carry no tiles and are written as zeros / -inf between items that do
+    B, L, Lk, Hq, Hkv, d, S, T, mask = 2, 6144, 3000, 16, 2, 128, 256, 128, [0, 1]
+    Q, K, V, dO = rand_inputs(B, L, Hq, Hkv, d, seed=11, Lk=Lk)
+    O, LSE = sa.seg_attn_fwd(Q, K, V, S, T, mask)
+    dQ, dK, dV = sa.seg_attn_bwd(Q, K, V, O, LSE, dO, S, T, mask)
+    sa.poll_status()
+    Oo, LSEo = oracle.fwd(f64(Q), f64(K), f64(V), S, T, mask)
+    ref = oracle.bwd(f64(Q), f64(K), f64(V), f64(dO), S, T, mask)
+    assert_fwd_close(O, LSE, Oo, LSEo, "many items")
+    assert_grads_close((dQ, dK, dV), ref, "many items")
+    g = Hq // Hkv
+    assert torch.isinf(LSE[:, :g, 3328:]).all() and torch.count_nonzero(O[:, 3328:, :g]) == 0   # local head: tail start >= 3000
+    assert torch.isfinite(LSE[:, g:]).all()                                                       # past-access head
+
+
 @pytest.mark.parametrize("B,L,Hq,Hkv,d,starts,T,mask,X", [
     (1, 1024, 4, 2, 128, [0, 200, 456, 457, 800], 100, [0, 1], 0),        # a one-token segment; tails longer than it
     (2, 700, 6, 3, 128, [0, 128, 256, 384, 512], 128, [2, 1, 0], 300),    # tile-aligned; a detached prefix
